@@ -1,0 +1,417 @@
+"""Benchmark of the fused Ulysses QKV prologue (QK RMSNorm + 2-D RoPE + the
+sequence-parallel -> head-parallel exchange, V first) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the prologue over one layer of the 21k-token workload
+(P=12 virtual ranks, S=21024, H=24, D=128, bf16), through the C ABI.  N > 1
+(torchrun) runs N independent replicas, one per GPU: the path has no exchange
+between devices in this build.  Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2604_14561_b200 import synth  # noqa: E402
+
+METRIC = "µs/layer and achieved HBM GB/s (% of B200 peak) for fused Ulysses QKV prologue"
+WORKLOAD = "qwen2304"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(cfg):
+    """Every element of Q, K, V read once and written once (bf16)."""
+    return 6 * cfg["S"] * cfg["H"] * cfg["D"] * 2
+
+
+# ----------------------------------------------------------------- clocks ---
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------- CPU oracle ---
+def oracle_sample(cfg, L, tokens):
+    """The oracle's full prologue on the first `tokens` tokens of the layer."""
+    import oracle
+    P, D = cfg["P"], cfg["D"]
+    sl = slice(0, tokens)
+    cs = oracle.rope_table_2d(L["pos"][sl], D, cfg["theta"])
+    q, k, v = (np.ascontiguousarray(L[n][sl]) for n in "qkv")
+    t0 = time.perf_counter()
+    oracle.prologue(q, k, v, L["wq"], L["wk"], cfg["eps"], cs, P)
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, on the host cores of this machine."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    cfg = synth.config(WORKLOAD)
+    tokens = cfg["S"] // cfg["P"]                    # one rank's shard: 1752 tokens, still P | tokens
+    assert tokens % cfg["P"] == 0
+    sub = dict(cfg, S=tokens)
+    E = tokens * cfg["H"] * cfg["D"]
+    L = {n: synth.normal_bf16(cfg["seed"], n, E).reshape(tokens, cfg["H"], cfg["D"]) for n in "qkv"}
+    L["wq"] = synth.normal_bf16(cfg["seed"], "wq", cfg["D"], 1.0, 0.1)
+    L["wk"] = synth.normal_bf16(cfg["seed"], "wk", cfg["D"], 1.0, 0.1)
+    L["pos"] = synth.positions(*cfg["grid"], cfg["n_text"])[:tokens]
+    for _ in range(args.warmup):
+        oracle_sample(sub, L, tokens)
+    t = [oracle_sample(sub, L, tokens) for _ in range(args.steps)]
+    total = sum(t)
+    bytes_per_step = algorithmic_bytes(sub)
+    gbs = bytes_per_step * args.steps / total / 1e9
+    sample = f"first {tokens} of {cfg['S']} tokens (one rank's shard) of the {WORKLOAD} layer per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "us_per_layer_extrapolated": 1e6 * total / args.steps * cfg["S"] / tokens,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 storage, fp32 arithmetic",
+        "data": "synthetic", "config": {"workload": WORKLOAD, "P": cfg["P"], "S": cfg["S"], "H": cfg["H"],
+                                        "D": cfg["D"], "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line, ensure_ascii=False))
+
+
+# --------------------------------------------------------------- GPU path ---
+def dev(a, torch):
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint16:
+        a = a.view(np.int16)
+    return torch.from_numpy(a).cuda()
+
+
+def time_steps(torch, fn, stream, steps, warmup, flush=None):
+    """CUDA events on `stream` around every step; returns per-step ms."""
+    for _ in range(warmup):
+        if flush is not None:
+            flush()
+        fn()
+    stream.synchronize()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev:
+        if flush is not None:
+            flush()
+        a.record(stream)
+        fn()
+        b.record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in ev]
+
+
+def max_over_ranks(ms, world, device):
+    """The slowest rank's time: every multi-GPU number is the max over ranks."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_gbs(step_bytes, world, ms_per_step):
+    """Whole-job throughput of `world` independent replicas (weak scaling)."""
+    return world * step_bytes / (ms_per_step * 1e-3) / 1e9
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2604_14561_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback for this path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    binding.lib()
+
+    cfg = synth.config(WORKLOAD)
+    P, S, H, D = cfg["P"], cfg["S"], cfg["H"], cfg["D"]
+    E = S * H * D
+    L = synth.make_layer(cfg)
+    q, k, v = (dev(L[n], torch) for n in "qkv")
+    wq, wk = dev(L["wq"], torch), dev(L["wk"], torch)
+    cs = torch.empty((S, D // 2, 2), dtype=torch.float32, device="cuda")
+    binding.rope_table_2d(cs, dev(L["pos"], torch), S, D, cfg["theta"])
+    qh, kh, vh = (torch.empty(E, dtype=torch.int16, device="cuda") for _ in range(3))
+    sq, sv = torch.cuda.Stream(), torch.cuda.Stream()
+    step_bytes = algorithmic_bytes(cfg)
+    peak, peak_kind = measured_peak()
+
+    def step(order):
+        binding.prologue(q, k, v, qh, kh, vh, wq, wk, cfg["eps"], cs, P, S, H, D, order=order,
+                         stream_qk=sq, stream_v=sv)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- headline: the V-first order, K steps back to back ------------------
+    for _ in range(max(args.warmup, 3)):
+        step(binding.V_FIRST)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record(sq)
+    for _ in range(args.steps):
+        step(binding.V_FIRST)
+    stop.record(sq)
+    barrier()
+    total_ms = start.elapsed_time(stop)
+    if rank == 0:
+        # keep the sampler running a little longer so that short runs still get samples under load
+        t_end = time.time() + 0.6
+        while time.time() < t_end:
+            step(binding.V_FIRST)
+        torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = max_over_ranks(total_ms, world, "cuda")
+    ms_per_step = total_ms / args.steps
+    value = aggregate_gbs(step_bytes, world, ms_per_step)
+
+    line = None
+    if rank == 0:
+        # ---- per-order detail, per-step events (this GPU only) --------------
+        orders = {}
+        for name, order in (("v_first", binding.V_FIRST), ("lump", binding.LUMP)):
+            ms = time_steps(torch, lambda: step(order), sq, args.steps, 3)
+            orders[name] = {"us_median": 1e3 * statistics.median(ms), "us_min": 1e3 * min(ms),
+                            "gbs_median": step_bytes / (statistics.median(ms) * 1e-3) / 1e9,
+                            "launches_per_step": 2 if order == binding.V_FIRST else 1}
+        # dominant kernel: move_rows_kernel, timed where one launch is the whole step (lump order)
+        lump_ms = statistics.mean(time_steps(torch, lambda: step(binding.LUMP), sq, args.steps, 3))
+        achieved = step_bytes / (lump_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "move_rows_kernel<LPR=16, mixed> (Q,K norm+RoPE+exchange and V exchange in one launch)",
+                    "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                    "frac": achieved / peak, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+                    "us_per_launch": 1e3 * lump_ms, "algorithmic_bytes_per_launch": step_bytes,
+                    "traffic": read_traffic_note()}
+
+        # ---- end to end: host buffers in, host buffers out ------------------
+        hin = [torch.from_numpy(L[n].view(np.int16)).pin_memory() for n in "qkv"]
+        hout = [torch.empty(E, dtype=torch.int16).pin_memory() for _ in range(3)]
+        dev_in = torch.empty(3 * E, dtype=torch.int16, device="cuda")
+        dev_out = torch.empty(3 * E, dtype=torch.int16, device="cuda")
+
+        def e2e_step():
+            binding.prologue_host(*hin, *hout, dev_in, dev_out, wq, wk, cfg["eps"], cs, P, S, H, D,
+                                  order=binding.V_FIRST, stream_qk=sq, stream_v=sv)
+        e2e_steps = max(3, min(args.steps, 10))
+        e2e_ms = statistics.mean(time_steps(torch, e2e_step, sq, e2e_steps, 2))
+        e2e = {"value": step_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
+               "steps": e2e_steps, "h2d_bytes_per_step": 3 * E * 2, "d2h_bytes_per_step": 3 * E * 2,
+               "api": "cocodiff_prologue_host (pinned host tensors in and out)"}
+        del hin, hout, dev_in, dev_out
+
+        per_config = other_configs(torch, binding, args)
+
+        # ---- the oracle on this machine's host cores, bounded sample ------------
+        import oracle
+        oracle.build()
+        tokens = S // P
+        sub = dict(cfg, S=tokens)
+        oracle_sample(sub, L, tokens)                       # warm the page cache / allocator
+        reps, spent = 0, 0.0
+        while spent < 10.0 and reps < 40:
+            spent += oracle_sample(sub, L, tokens)
+            reps += 1
+        cpu_gbs = algorithmic_bytes(sub) * reps / spent / 1e9
+        cpu = {"value": cpu_gbs, "unit": "GB/s", "cores": 1, "kind": "oracle",
+               "ms_per_layer_extrapolated": 1e3 * spent / reps * S / tokens,
+               "sample": f"{reps} passes over the first {tokens} of {S} tokens (one rank's shard) of the same layer"}
+
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "us_per_layer": 1e3 * ms_per_step,
+            "frac_of_nominal_8000": value / world / NOMINAL_HBM_GBS, "frac_of_measured_copy": value / world / peak,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 storage, fp32 arithmetic", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "P": P, "S": S, "H": H, "D": D, "order": "v_first",
+                       "algorithmic_bytes_per_step": step_bytes, "l2": "inputs and outputs (775 MB per step) exceed the 126 MB L2",
+                       "replicas": world},
+            "gpu_launches": 2 * args.steps,
+            "clocks": clocks, "orders": orders, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+            "per_config": per_config,
+        }
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line, ensure_ascii=False))
+
+
+def read_traffic_note():
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if present."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f).get("move_rows_mixed_qwen2304_bytes_per_launch")
+    except Exception:
+        return None
+
+
+def other_configs(torch, binding, args):
+    """µs/layer and GB/s of the other synthetic workloads, L2 flushed between
+    iterations (they fit in the 126 MB L2), plus the selective step of the
+    temporal workload."""
+    out = {}
+    scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    sq, sv = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def flush():
+        with torch.cuda.stream(sq):
+            scratch.zero_()
+
+    iters = max(10, min(args.steps, 50))
+    for name in ("tiny", "sd3", "qwen768", "temporal"):
+        cfg = synth.config(name)
+        P, S, H, D = cfg["P"], cfg["S"], cfg["H"], cfg["D"]
+        E = S * H * D
+        L = synth.make_layer(cfg)
+        q, k, v = (dev(L[n], torch) for n in "qkv")
+        wq, wk = dev(L["wq"], torch), dev(L["wk"], torch)
+        cs = torch.empty((S, D // 2, 2), dtype=torch.float32, device="cuda")
+        binding.rope_table_2d(cs, dev(L["pos"], torch), S, D, cfg["theta"])
+        qh, kh, vh = (torch.empty(E, dtype=torch.int16, device="cuda") for _ in range(3))
+
+        def full():
+            binding.prologue(q, k, v, qh, kh, vh, wq, wk, cfg["eps"], cs, P, S, H, D,
+                             order=binding.V_FIRST, stream_qk=sq, stream_v=sv)
+        cold = time_steps(torch, full, sq, iters, 3, flush=flush)
+        warm = time_steps(torch, full, sq, iters, 3)
+        b = algorithmic_bytes(cfg)
+        out[name] = {"bytes": b, "us_cold_l2": 1e3 * statistics.median(cold),
+                     "gbs_cold_l2": b / (statistics.median(cold) * 1e-3) / 1e9,
+                     "us_warm_l2": 1e3 * statistics.median(warm)}
+        if name != "temporal":
+            continue
+        # selective step: metric + selection + V compaction, K/Q compaction (norm + RoPE fused), three scatters
+        T, r, n_groups = cfg["T"], cfg["r"], cfg["n_groups"]
+        n = S // T
+        seq_rng = np.random.default_rng(0)
+        hot = np.sort(seq_rng.choice(n, int(np.ceil(cfg["frac_large"] * n)), replace=False))
+        cur = synth.bf16_bits_to_f32(L["v"]).reshape(n, -1).copy()
+        cur[hot] += synth.normal_f32(9, "bump", len(hot) * cur.shape[1], 0.0, cfg["sigma_large"]).reshape(len(hot), -1)
+        cur_v = dev(synth.f32_to_bf16_bits(cur).reshape(S, H, D), torch)
+        ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        metric = torch.zeros(n, dtype=torch.int64, device="cuda")
+        mask = torch.zeros(n, dtype=torch.uint8, device="cuda")
+        idx = torch.zeros(n, dtype=torch.int32, device="cuda")
+        na = torch.zeros(1, dtype=torch.int32, device="cuda")
+        comp = [torch.empty(E, dtype=torch.int16, device="cuda") for _ in range(3)]
+
+        def selective():
+            binding.vmajor_select_compact(v, cur_v, P, S, H, D, T, r, n_groups, metric, mask, idx, na, comp[2],
+                                          ws, ws_bytes, stream=sq)
+            binding.pack_active(k, wk, cfg["eps"], cs, idx, na, comp[1], P, S, H, D, T, stream=sq)
+            binding.pack_active(q, wq, cfg["eps"], cs, idx, na, comp[0], P, S, H, D, T, stream=sq)
+            binding.unpack(comp[2], idx, na, vh, P, S, H, D, T, stream=sq)
+            binding.unpack(comp[1], idx, na, kh, P, S, H, D, T, stream=sq)
+            binding.unpack(comp[0], idx, na, qh, P, S, H, D, T, stream=sq)
+        cold = time_steps(torch, selective, sq, iters, 3, flush=flush)
+        n_act = int(na.item())
+        tile = T * H * D * 2
+        sb = 2 * E * 2 + 3 * 2 * n_act * tile + 3 * 2 * n_act * tile
+        out["temporal_selective_step"] = {"n_active": n_act, "n_units": n, "bytes": sb,
+                                          "us_cold_l2": 1e3 * statistics.median(cold),
+                                          "gbs_cold_l2": sb / (statistics.median(cold) * 1e-3) / 1e9,
+                                          "launches_per_step": 8}
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

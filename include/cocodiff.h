@@ -1,0 +1,168 @@
+/*
+ * libcocodiff - the per-layer Ulysses attention prologue of CoCoDiff on one
+ * NVIDIA B200 (sm_100a): QK RMSNorm + 2-D RoPE, the sequence-parallel ->
+ * head-parallel exchange issued V-first, and V-Major selection / compaction /
+ * reconstruction.  The P ranks are virtual shards of one device's memory, so
+ * the all-to-all is a device-local permutation.
+ *
+ * Conventions for every entry point
+ *   - Returns 0 (COCODIFF_OK) or a negative cocodiff_status.  On an error
+ *     nothing has been enqueued.
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned
+ *     by the caller.  The library allocates no device memory, never
+ *     synchronises the device and enqueues only on the streams it is given
+ *     (void* = cudaStream_t, NULL = the default stream).  Calls return as soon
+ *     as the work is enqueued.
+ *   - bf16 tensors are passed as uint16_t bit patterns, row-major, last index
+ *     fastest, and must be 16-byte aligned.  Head dimension D is one of
+ *     32, 64, 128, 256.
+ *   - Layouts:  SEQ  = [P][S/P][H][D] == [S][H][D]  (rank p owns tokens
+ *                      [p*S/P, (p+1)*S/P): the sequence-parallel layout)
+ *               HEAD = [P][H/P][S][D] == [H][S][D]  (rank p owns heads
+ *                      [p*H/P, (p+1)*H/P): the head-parallel layout)
+ *     (Section II-A of the paper.)  P must divide S and H, and P <= H: one
+ *     head per rank is the Ulysses limit (Section IV-B).
+ *   - A selection unit is T consecutive tokens of one source rank, all heads
+ *     (T = 1 is the paper's per-token rule); T must divide S/P.
+ *     COMPACT = [H][n_active][T][D] == [P][H/P][n_active*T][D]: what each
+ *     destination rank receives when only the active units are sent, source
+ *     ranks concatenated in rank order (ascending unit index).
+ */
+#ifndef COCODIFF_H
+#define COCODIFF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    COCODIFF_OK = 0,
+    COCODIFF_INVALID_ARG = -1,         /* null pointer, P < 1, r outside [0,1], bad enum          */
+    COCODIFF_BAD_SHAPE = -2,           /* P does not divide S or H, P > H, unsupported D, T, groups */
+    COCODIFF_MISALIGNED = -3,          /* a tensor pointer is not 16-byte aligned                  */
+    COCODIFF_WORKSPACE_TOO_SMALL = -4,
+    COCODIFF_CUDA_ERROR = -5,          /* a launch or copy failed; see cocodiff_last_cuda_error()  */
+    COCODIFF_ALIASING = -6             /* input and output overlap where that is not allowed       */
+} cocodiff_status;
+
+/* Order of issue of the three exchanges (Section III-C, "V-First Scheduling").
+ * LUMP: Q, K and V leave together in one launch on stream_qk (the flat order).
+ * V_FIRST: V's exchange is launched first, on stream_v, and runs beside the
+ * norm + RoPE + exchange of Q and K on stream_qk.  Results are identical. */
+typedef enum { COCODIFF_LUMP = 0, COCODIFF_V_FIRST = 1 } cocodiff_order;
+
+const char *cocodiff_status_string(int status);
+int cocodiff_version(void);
+/* cudaError_t of the most recent COCODIFF_CUDA_ERROR on the calling thread (0 if none). */
+int cocodiff_last_cuda_error(void);
+
+/* RoPE angle table (Section II-B, "Rotary position embeddings"; axial 2-D form).
+ * cs[s][p] = (cos, sin) of pos[s][axis] * theta^(-2i/(D/2)) with axis = p / (D/4),
+ * i = p % (D/4): the first D/4 pairs (dimensions [0, D/2)) rotate with the row
+ * position, the last D/4 with the column position.  cs: [S][D/2][2] float out;
+ * pos: [S][2] int32 (row, col).  Evaluated in double on the device, rounded to
+ * float.  Built once per resolution, not per layer. */
+int cocodiff_rope_table_2d(float *cs, const int32_t *pos, int S, int D, double theta, void *stream);
+
+/* QK normalisation + RoPE alone (Section II-B), SEQ in -> SEQ out.
+ * y = RoPE(x * rsqrt(mean_D(x^2) + eps) * w), per (token, head), fp32 arithmetic,
+ * one round-to-nearest-even to bf16.  Pair (2p, 2p+1) is rotated by cs[s][p].
+ * q/k may be NULL to skip that tensor; out == in (same tensor) is allowed,
+ * any other overlap is COCODIFF_ALIASING.  wq, wk: [D] bf16.  cs may be NULL
+ * (no rotation). */
+int cocodiff_qk_norm_rope(const uint16_t *q, const uint16_t *k, uint16_t *q_out, uint16_t *k_out,
+                          const uint16_t *wq, const uint16_t *wk, float eps, const float *cs,
+                          int S, int H, int D, void *stream);
+
+/* The Ulysses exchange alone (Section II-A): SEQ -> HEAD, bit-exact move.
+ * Any of the (x, x_head) pairs may be NULL/NULL to skip it.  With V_FIRST and
+ * stream_v != stream_qk, stream_v first waits for the work already enqueued
+ * on stream_qk, and stream_qk afterwards waits for V: to the caller the call
+ * is ordered on stream_qk. */
+int cocodiff_ulysses_a2a(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                         uint16_t *q_head, uint16_t *k_head, uint16_t *v_head,
+                         int P, int S, int H, int D, cocodiff_order order,
+                         void *stream_qk, void *stream_v);
+
+/* The second all-to-all of Section II-A: HEAD -> SEQ, bit-exact move. */
+int cocodiff_ulysses_a2a_inverse(const uint16_t *q_head, const uint16_t *k_head, const uint16_t *v_head,
+                                 uint16_t *q, uint16_t *k, uint16_t *v,
+                                 int P, int S, int H, int D, void *stream);
+
+/* The fused prologue of one layer, full exchange (Sections II-B, II-A, III-C):
+ * every (token, head) row of Q and K is read once, normalised, rotated and
+ * written straight into its HEAD slot; V is moved untouched, first.  Stream
+ * semantics as for cocodiff_ulysses_a2a.  All six tensors are required. */
+int cocodiff_prologue(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                      uint16_t *q_head, uint16_t *k_head, uint16_t *v_head,
+                      const uint16_t *wq, const uint16_t *wk, float eps, const float *cs,
+                      int P, int S, int H, int D, cocodiff_order order,
+                      void *stream_qk, void *stream_v);
+
+/* The same prologue for HOST tensors: q, k, v and the three results are host
+ * pointers (pinned memory makes the copies asynchronous); dev_in and dev_out
+ * are caller-owned device staging buffers of 3*S*H*D bf16 each.  V is copied,
+ * exchanged and copied back on stream_v while Q and K follow on stream_qk
+ * (V_FIRST), or everything runs on stream_qk (LUMP).  wq, wk, cs stay device
+ * pointers.  On return stream_qk is ordered after all of it. */
+int cocodiff_prologue_host(const uint16_t *q_host, const uint16_t *k_host, const uint16_t *v_host,
+                           uint16_t *q_head_host, uint16_t *k_head_host, uint16_t *v_head_host,
+                           uint16_t *dev_in, uint16_t *dev_out,
+                           const uint16_t *wq, const uint16_t *wk, float eps, const float *cs,
+                           int P, int S, int H, int D, cocodiff_order order,
+                           void *stream_qk, void *stream_v);
+
+/* V-Major active-projection selection (Section III-D, "Active projection
+ * selection") and compaction of V.
+ *   metric[u] = sum over the unit's T*H*D elements of fix(|cur - prev|), where
+ *     the difference is one fp32 subtraction and fix(d) = min(trunc(d * 2^16),
+ *     2^32 - 1) (NaN -> 2^32 - 1): an integer L1 distance, independent of the
+ *     order of accumulation.
+ *   The n = S/T units form n_groups contiguous groups of g units (1 = one
+ *     global decision, P/2 = the paper's per-GPU scope, P = per rank).  In each
+ *     group the floor(r * g) units smallest by (metric, index) are cached
+ *     (mask 0), the others active (mask 1).
+ *   idx[0 .. n_active) = the active units, ascending; n_active is written to
+ *     device memory (the host can compute it: n - n_groups * floor(r * g)).
+ *   v_compact, if not NULL: COMPACT layout of the active units of cur_v
+ *     (capacity S*H*D elements).
+ * prev_v is only read: which step it holds is the caller's policy.
+ * workspace: cocodiff_vmajor_workspace_bytes() bytes of scratch, 256-byte
+ * aligned; contents are undefined on entry and on exit (the call clears what
+ * it needs).  It holds the per-unit accumulators and the block ticket of the
+ * fused metric + selection kernel.  Concurrent calls need distinct workspaces. */
+size_t cocodiff_vmajor_workspace_bytes(int P, int S, int H, int D, int T);
+int cocodiff_vmajor_select_compact(const uint16_t *prev_v, const uint16_t *cur_v,
+                                   int P, int S, int H, int D, int T, double r, int n_groups,
+                                   uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
+                                   uint16_t *v_compact,
+                                   void *workspace, size_t workspace_bytes, void *stream);
+
+/* Selection alone from a given metric array (the rule of the same passage);
+ * used by the call above and exposed for tests and for callers that keep their
+ * own metric. */
+int cocodiff_vmajor_select(const uint64_t *metric, int n, double r, int n_groups,
+                           uint8_t *mask, int32_t *idx, int32_t *n_active, void *stream);
+
+/* Extraction of the active units of one tensor into COMPACT (Section III-D,
+ * "Selective communication in TAPA").  w != NULL: the rows are normalised and
+ * rotated on the way (Q, K); w == NULL: plain move (V).  idx and n_active are
+ * read on the device, so no host round trip separates selection and packing.
+ * x_compact capacity: S*H*D elements. */
+int cocodiff_pack_active(const uint16_t *x, const uint16_t *w, float eps, const float *cs,
+                         const int32_t *idx, const int32_t *n_active, uint16_t *x_compact,
+                         int P, int S, int H, int D, int T, void *stream);
+
+/* Receiver-side reconstruction (Section III-D, "Post-Phase 2"): indexed scatter
+ * x_cache[h][idx[a]*T + j][:] = x_compact[h][a][j][:]; all other rows of the
+ * cached HEAD tensor keep their bits. */
+int cocodiff_unpack(const uint16_t *x_compact, const int32_t *idx, const int32_t *n_active,
+                    uint16_t *x_cache, int P, int S, int H, int D, int T, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COCODIFF_H */

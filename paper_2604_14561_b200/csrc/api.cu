@@ -1,0 +1,441 @@
+// C ABI of libcocodiff: argument validation, stream / event wiring and the
+// launch plan of every entry point declared in include/cocodiff.h.  No kernel
+// lives here and no device memory is allocated here.
+#include <cmath>
+#include <cstring>
+
+#include "../../include/cocodiff.h"
+#include "common.cuh"
+
+using namespace cocodiff;
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+int cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int)e;
+    return COCODIFF_CUDA_ERROR;
+}
+
+#define CK(expr)                                       \
+    do {                                               \
+        const cudaError_t e__ = (expr);                \
+        if (e__ != cudaSuccess) return cuda_fail(e__); \
+    } while (0)
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool overlap(const void *a, size_t na, const void *b, size_t nb) {
+    if (!a || !b || na == 0 || nb == 0) return false;
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return x < y + nb && y < x + na;
+}
+
+bool supported_d(int D) { return D == 32 || D == 64 || D == 128 || D == 256; }
+
+int check_shape(int P, int S, int H, int D) {
+    if (P < 1 || S < 0 || H < 1) return COCODIFF_INVALID_ARG;
+    if (!supported_d(D)) return COCODIFF_BAD_SHAPE;
+    if (S % P != 0 || H % P != 0 || P > H) return COCODIFF_BAD_SHAPE;
+    if ((long long)S * H * D > (1LL << 40)) return COCODIFF_BAD_SHAPE;
+    return COCODIFF_OK;
+}
+
+int check_unit(int P, int S, int T) {
+    if (T < 1) return COCODIFF_INVALID_ARG;
+    if ((S / P) % T != 0) return COCODIFF_BAD_SHAPE;
+    return COCODIFF_OK;
+}
+
+// Two timing-less events per (thread, device) for the fork / join of the V stream.
+struct ForkJoin {
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
+constexpr int kMaxDevices = 64;
+thread_local ForkJoin g_events[kMaxDevices];
+
+int get_events(ForkJoin **out) {
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return COCODIFF_INVALID_ARG;
+    ForkJoin &fj = g_events[dev];
+    if (!fj.fork) {
+        CK(cudaEventCreateWithFlags(&fj.fork, cudaEventDisableTiming));
+        CK(cudaEventCreateWithFlags(&fj.join, cudaEventDisableTiming));
+    }
+    *out = &fj;
+    return COCODIFF_OK;
+}
+
+MoveParams seq_to_head(int S, int H, int D) {
+    MoveParams p;
+    std::memset(&p, 0, sizeof p);
+    p.n_slots = S;
+    p.H = H;
+    p.src_tok = (long long)H * D;
+    p.src_head = D;
+    p.dst_tok = D;
+    p.dst_head = (long long)S * D;
+    p.map = MAP_FULL;
+    p.T = 1;
+    return p;
+}
+
+// Shared by cocodiff_ulysses_a2a (no weights) and cocodiff_prologue.
+int exchange(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *qh, uint16_t *kh,
+             uint16_t *vh, const uint16_t *wq, const uint16_t *wk, float eps, const float *cs, int S,
+             int H, int D, int order, cudaStream_t sq, cudaStream_t sv) {
+    MoveParams base = seq_to_head(S, H, D);
+    base.cs = cs;
+    base.eps = eps;
+    const bool two_streams = order == COCODIFF_V_FIRST && sv != sq && v != nullptr && (q || k);
+    if (order == COCODIFF_LUMP || !two_streams) {
+        // one launch; V's blocks come first in the grid
+        MoveParams p = base;
+        if (v) p.job[p.njobs++] = MoveJob{v, vh, nullptr};
+        if (q) p.job[p.njobs++] = MoveJob{q, qh, wq};
+        if (k) p.job[p.njobs++] = MoveJob{k, kh, wk};
+        if (p.njobs == 0) return COCODIFF_OK;
+        CK(launch_move(p, D, sq));
+        return COCODIFF_OK;
+    }
+    ForkJoin *fj = nullptr;
+    const int rc = get_events(&fj);
+    if (rc != COCODIFF_OK) return rc;
+    CK(cudaEventRecord(fj->fork, sq));
+    CK(cudaStreamWaitEvent(sv, fj->fork, 0));
+    MoveParams pv = base;
+    pv.job[pv.njobs++] = MoveJob{v, vh, nullptr};
+    CK(launch_move(pv, D, sv));
+    MoveParams pqk = base;
+    if (q) pqk.job[pqk.njobs++] = MoveJob{q, qh, wq};
+    if (k) pqk.job[pqk.njobs++] = MoveJob{k, kh, wk};
+    CK(launch_move(pqk, D, sq));
+    CK(cudaEventRecord(fj->join, sv));
+    CK(cudaStreamWaitEvent(sq, fj->join, 0));
+    return COCODIFF_OK;
+}
+
+int check_pairs(const uint16_t *const in[3], uint16_t *const out[3], size_t bytes) {
+    for (int i = 0; i < 3; ++i) {
+        if ((in[i] == nullptr) != (out[i] == nullptr)) return COCODIFF_INVALID_ARG;
+        if (!aligned16(in[i]) || !aligned16(out[i])) return COCODIFF_MISALIGNED;
+    }
+    for (int i = 0; i < 3; ++i)
+        for (int j = 0; j < 3; ++j) {
+            if (overlap(in[i], bytes, out[j], bytes)) return COCODIFF_ALIASING;
+            if (i < j && overlap(out[i], bytes, out[j], bytes)) return COCODIFF_ALIASING;
+        }
+    return COCODIFF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *cocodiff_status_string(int status) {
+    switch (status) {
+        case COCODIFF_OK: return "ok";
+        case COCODIFF_INVALID_ARG: return "invalid argument";
+        case COCODIFF_BAD_SHAPE: return "unsupported shape";
+        case COCODIFF_MISALIGNED: return "pointer not 16-byte aligned";
+        case COCODIFF_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case COCODIFF_CUDA_ERROR: return "CUDA error";
+        case COCODIFF_ALIASING: return "input and output overlap";
+        default: return "unknown status";
+    }
+}
+
+int cocodiff_version(void) { return 100; }
+
+int cocodiff_last_cuda_error(void) { return g_last_cuda_error; }
+
+int cocodiff_rope_table_2d(float *cs, const int32_t *pos, int S, int D, double theta, void *stream) {
+    if (!cs || !pos || S < 0 || !(theta > 0.0)) return COCODIFF_INVALID_ARG;
+    if (!supported_d(D)) return COCODIFF_BAD_SHAPE;
+    if (!aligned16(cs) || (reinterpret_cast<uintptr_t>(pos) & 3u)) return COCODIFF_MISALIGNED;
+    CK(launch_rope_table(cs, pos, S, D, theta, (cudaStream_t)stream));
+    return COCODIFF_OK;
+}
+
+int cocodiff_qk_norm_rope(const uint16_t *q, const uint16_t *k, uint16_t *q_out, uint16_t *k_out,
+                          const uint16_t *wq, const uint16_t *wk, float eps, const float *cs, int S,
+                          int H, int D, void *stream) {
+    if (S < 0 || H < 1 || !(eps >= 0.f)) return COCODIFF_INVALID_ARG;
+    if (!supported_d(D) || (long long)S * H * D > (1LL << 40)) return COCODIFF_BAD_SHAPE;
+    if ((q == nullptr) != (q_out == nullptr) || (k == nullptr) != (k_out == nullptr)) return COCODIFF_INVALID_ARG;
+    if ((q && !wq) || (k && !wk)) return COCODIFF_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(q_out) || !aligned16(k_out) || !aligned16(wq) ||
+        !aligned16(wk) || !aligned16(cs))
+        return COCODIFF_MISALIGNED;
+    const size_t bytes = (size_t)S * H * D * 2;
+    if ((q_out != q && overlap(q, bytes, q_out, bytes)) || (k_out != k && overlap(k, bytes, k_out, bytes)) ||
+        overlap(q, bytes, k_out, bytes) || overlap(k, bytes, q_out, bytes) || overlap(q_out, bytes, k_out, bytes))
+        return COCODIFF_ALIASING;
+    MoveParams p;
+    std::memset(&p, 0, sizeof p);
+    p.n_slots = S;
+    p.H = H;
+    p.src_tok = p.dst_tok = (long long)H * D;
+    p.src_head = p.dst_head = D;
+    p.map = MAP_FULL;
+    p.T = 1;
+    p.cs = cs;
+    p.eps = eps;
+    if (q) p.job[p.njobs++] = MoveJob{q, q_out, wq};
+    if (k) p.job[p.njobs++] = MoveJob{k, k_out, wk};
+    if (p.njobs == 0) return COCODIFF_OK;
+    CK(launch_move(p, D, (cudaStream_t)stream));
+    return COCODIFF_OK;
+}
+
+int cocodiff_ulysses_a2a(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *q_head,
+                         uint16_t *k_head, uint16_t *v_head, int P, int S, int H, int D,
+                         cocodiff_order order, void *stream_qk, void *stream_v) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    if (order != COCODIFF_LUMP && order != COCODIFF_V_FIRST) return COCODIFF_INVALID_ARG;
+    const uint16_t *in[3] = {q, k, v};
+    uint16_t *out[3] = {q_head, k_head, v_head};
+    rc = check_pairs(in, out, (size_t)S * H * D * 2);
+    if (rc) return rc;
+    return exchange(q, k, v, q_head, k_head, v_head, nullptr, nullptr, 0.f, nullptr, S, H, D, order,
+                    (cudaStream_t)stream_qk, (cudaStream_t)stream_v);
+}
+
+int cocodiff_ulysses_a2a_inverse(const uint16_t *q_head, const uint16_t *k_head, const uint16_t *v_head,
+                                 uint16_t *q, uint16_t *k, uint16_t *v, int P, int S, int H, int D,
+                                 void *stream) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    const uint16_t *in[3] = {q_head, k_head, v_head};
+    uint16_t *out[3] = {q, k, v};
+    rc = check_pairs(in, out, (size_t)S * H * D * 2);
+    if (rc) return rc;
+    MoveParams p;
+    std::memset(&p, 0, sizeof p);
+    p.n_slots = S;
+    p.H = H;
+    p.src_tok = D;
+    p.src_head = (long long)S * D;
+    p.dst_tok = (long long)H * D;
+    p.dst_head = D;
+    p.map = MAP_FULL;
+    p.T = 1;
+    for (int i = 2; i >= 0; --i)
+        if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr};
+    if (p.njobs == 0) return COCODIFF_OK;
+    CK(launch_move(p, D, (cudaStream_t)stream));
+    return COCODIFF_OK;
+}
+
+int cocodiff_prologue(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *q_head,
+                      uint16_t *k_head, uint16_t *v_head, const uint16_t *wq, const uint16_t *wk,
+                      float eps, const float *cs, int P, int S, int H, int D, cocodiff_order order,
+                      void *stream_qk, void *stream_v) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    if (order != COCODIFF_LUMP && order != COCODIFF_V_FIRST) return COCODIFF_INVALID_ARG;
+    if (!q || !k || !v || !q_head || !k_head || !v_head || !wq || !wk || !cs || !(eps >= 0.f))
+        return COCODIFF_INVALID_ARG;
+    if (!aligned16(wq) || !aligned16(wk) || !aligned16(cs)) return COCODIFF_MISALIGNED;
+    const uint16_t *in[3] = {q, k, v};
+    uint16_t *out[3] = {q_head, k_head, v_head};
+    rc = check_pairs(in, out, (size_t)S * H * D * 2);
+    if (rc) return rc;
+    return exchange(q, k, v, q_head, k_head, v_head, wq, wk, eps, cs, S, H, D, order,
+                    (cudaStream_t)stream_qk, (cudaStream_t)stream_v);
+}
+
+int cocodiff_prologue_host(const uint16_t *q_host, const uint16_t *k_host, const uint16_t *v_host,
+                           uint16_t *q_head_host, uint16_t *k_head_host, uint16_t *v_head_host,
+                           uint16_t *dev_in, uint16_t *dev_out, const uint16_t *wq, const uint16_t *wk,
+                           float eps, const float *cs, int P, int S, int H, int D, cocodiff_order order,
+                           void *stream_qk, void *stream_v) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    if (order != COCODIFF_LUMP && order != COCODIFF_V_FIRST) return COCODIFF_INVALID_ARG;
+    if (!q_host || !k_host || !v_host || !q_head_host || !k_head_host || !v_head_host || !dev_in ||
+        !dev_out || !wq || !wk || !cs || !(eps >= 0.f))
+        return COCODIFF_INVALID_ARG;
+    if (!aligned16(dev_in) || !aligned16(dev_out) || !aligned16(wq) || !aligned16(wk) || !aligned16(cs))
+        return COCODIFF_MISALIGNED;
+    const size_t E = (size_t)S * H * D, bytes = E * 2;
+    if (overlap(dev_in, 3 * bytes, dev_out, 3 * bytes)) return COCODIFF_ALIASING;
+    cudaStream_t sq = (cudaStream_t)stream_qk, sv = (cudaStream_t)stream_v;
+    if (order == COCODIFF_LUMP) sv = sq;
+    uint16_t *dq = dev_in, *dk = dev_in + E, *dv = dev_in + 2 * E;
+    uint16_t *oq = dev_out, *ok = dev_out + E, *ov = dev_out + 2 * E;
+    MoveParams base = seq_to_head(S, H, D);
+    base.cs = cs;
+    base.eps = eps;
+    ForkJoin *fj = nullptr;
+    if (sv != sq) {
+        rc = get_events(&fj);
+        if (rc) return rc;
+        CK(cudaEventRecord(fj->fork, sq));
+        CK(cudaStreamWaitEvent(sv, fj->fork, 0));
+    }
+    // V first: copy in, exchange, copy out on its own stream
+    CK(cudaMemcpyAsync(dv, v_host, bytes, cudaMemcpyHostToDevice, sv));
+    MoveParams pv = base;
+    pv.job[pv.njobs++] = MoveJob{dv, ov, nullptr};
+    CK(launch_move(pv, D, sv));
+    CK(cudaMemcpyAsync(v_head_host, ov, bytes, cudaMemcpyDeviceToHost, sv));
+    CK(cudaMemcpyAsync(dq, q_host, bytes, cudaMemcpyHostToDevice, sq));
+    CK(cudaMemcpyAsync(dk, k_host, bytes, cudaMemcpyHostToDevice, sq));
+    MoveParams pqk = base;
+    pqk.job[pqk.njobs++] = MoveJob{dq, oq, wq};
+    pqk.job[pqk.njobs++] = MoveJob{dk, ok, wk};
+    CK(launch_move(pqk, D, sq));
+    CK(cudaMemcpyAsync(q_head_host, oq, bytes, cudaMemcpyDeviceToHost, sq));
+    CK(cudaMemcpyAsync(k_head_host, ok, bytes, cudaMemcpyDeviceToHost, sq));
+    if (sv != sq) {
+        CK(cudaEventRecord(fj->join, sv));
+        CK(cudaStreamWaitEvent(sq, fj->join, 0));
+    }
+    return COCODIFF_OK;
+}
+
+size_t cocodiff_vmajor_workspace_bytes(int P, int S, int H, int D, int T) {
+    (void)H;
+    (void)D;
+    if (P < 1 || T < 1 || S < 0) return 0;
+    const size_t n = (size_t)(S / T);
+    return ((n * 8 + 255) / 256) * 256 + 256;  // accumulators, then the ticket
+}
+
+int cocodiff_vmajor_select(const uint64_t *metric, int n, double r, int n_groups, uint8_t *mask,
+                           int32_t *idx, int32_t *n_active, void *stream) {
+    if (!metric || !mask || !idx || !n_active || n < 0 || n_groups < 1 || !(r >= 0.0 && r <= 1.0))
+        return COCODIFF_INVALID_ARG;
+    if (n % n_groups != 0) return COCODIFF_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(metric) & 7u) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
+        (reinterpret_cast<uintptr_t>(n_active) & 3u))
+        return COCODIFF_MISALIGNED;
+    SelectParams sp;
+    sp.metric = reinterpret_cast<const unsigned long long *>(metric);
+    sp.n = n;
+    sp.n_groups = n_groups;
+    sp.g = n / n_groups;
+    sp.n_cached = (int)std::floor(r * (double)sp.g);
+    sp.mask = mask;
+    sp.idx = idx;
+    sp.n_active = n_active;
+    CK(launch_select(sp, (cudaStream_t)stream));
+    return COCODIFF_OK;
+}
+
+int cocodiff_vmajor_select_compact(const uint16_t *prev_v, const uint16_t *cur_v, int P, int S, int H,
+                                   int D, int T, double r, int n_groups, uint64_t *metric, uint8_t *mask,
+                                   int32_t *idx, int32_t *n_active, uint16_t *v_compact, void *workspace,
+                                   size_t workspace_bytes, void *stream) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    rc = check_unit(P, S, T);
+    if (rc) return rc;
+    if (!prev_v || !cur_v || !metric || !mask || !idx || !n_active || !workspace || n_groups < 1 ||
+        !(r >= 0.0 && r <= 1.0))
+        return COCODIFF_INVALID_ARG;
+    const int n = S / T;
+    if (n % n_groups != 0) return COCODIFF_BAD_SHAPE;
+    if (!aligned16(prev_v) || !aligned16(cur_v) || !aligned16(v_compact) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255u) || (reinterpret_cast<uintptr_t>(metric) & 7u) ||
+        (reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(n_active) & 3u))
+        return COCODIFF_MISALIGNED;
+    const size_t need = cocodiff_vmajor_workspace_bytes(P, S, H, D, T);
+    if (workspace_bytes < need) return COCODIFF_WORKSPACE_TOO_SMALL;
+    const size_t bytes = (size_t)S * H * D * 2;
+    if (overlap(cur_v, bytes, v_compact, bytes) || overlap(prev_v, bytes, v_compact, bytes))
+        return COCODIFF_ALIASING;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    MetricParams mp;
+    std::memset(&mp, 0, sizeof mp);
+    mp.prev = reinterpret_cast<const uint4 *>(prev_v);
+    mp.cur = reinterpret_cast<const uint4 *>(cur_v);
+    mp.acc = reinterpret_cast<unsigned long long *>(workspace);
+    mp.ticket = reinterpret_cast<unsigned int *>(reinterpret_cast<char *>(workspace) + (need - 256));
+    mp.metric = reinterpret_cast<unsigned long long *>(metric);
+    mp.unit_vecs = (long long)T * H * D / 8;
+    mp.chunk_vecs = 512;
+    mp.chunks_per_unit = (int)((mp.unit_vecs + mp.chunk_vecs - 1) / mp.chunk_vecs);
+    mp.n_units = n;
+    mp.sel.metric = mp.metric;
+    mp.sel.n = n;
+    mp.sel.n_groups = n_groups;
+    mp.sel.g = n / n_groups;
+    mp.sel.n_cached = (int)std::floor(r * (double)mp.sel.g);
+    mp.sel.mask = mask;
+    mp.sel.idx = idx;
+    mp.sel.n_active = n_active;
+    CK(cudaMemsetAsync(workspace, 0, need, st));
+    CK(launch_metric_select(mp, st));
+    if (v_compact)
+        return cocodiff_pack_active(cur_v, nullptr, 0.f, nullptr, idx, n_active, v_compact, P, S, H, D, T, stream);
+    return COCODIFF_OK;
+}
+
+int cocodiff_pack_active(const uint16_t *x, const uint16_t *w, float eps, const float *cs,
+                         const int32_t *idx, const int32_t *n_active, uint16_t *x_compact, int P, int S,
+                         int H, int D, int T, void *stream) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    rc = check_unit(P, S, T);
+    if (rc) return rc;
+    if (!x || !idx || !n_active || !x_compact || !(eps >= 0.f)) return COCODIFF_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(x_compact) || !aligned16(w) || !aligned16(cs) ||
+        (reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(n_active) & 3u))
+        return COCODIFF_MISALIGNED;
+    const size_t bytes = (size_t)S * H * D * 2;
+    if (overlap(x, bytes, x_compact, bytes)) return COCODIFF_ALIASING;
+    MoveParams p;
+    std::memset(&p, 0, sizeof p);
+    p.n_slots = S;
+    p.H = H;
+    p.src_tok = (long long)H * D;
+    p.src_head = D;
+    p.dst_tok = D;
+    p.dst_head = COMPACT_STRIDE;
+    p.map = MAP_GATHER;
+    p.T = T;
+    p.idx = idx;
+    p.n_active = n_active;
+    p.cs = w ? cs : nullptr;
+    p.eps = eps;
+    p.job[p.njobs++] = MoveJob{x, x_compact, w};
+    CK(launch_move(p, D, (cudaStream_t)stream));
+    return COCODIFF_OK;
+}
+
+int cocodiff_unpack(const uint16_t *x_compact, const int32_t *idx, const int32_t *n_active,
+                    uint16_t *x_cache, int P, int S, int H, int D, int T, void *stream) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    rc = check_unit(P, S, T);
+    if (rc) return rc;
+    if (!x_compact || !idx || !n_active || !x_cache) return COCODIFF_INVALID_ARG;
+    if (!aligned16(x_compact) || !aligned16(x_cache) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
+        (reinterpret_cast<uintptr_t>(n_active) & 3u))
+        return COCODIFF_MISALIGNED;
+    const size_t bytes = (size_t)S * H * D * 2;
+    if (overlap(x_compact, bytes, x_cache, bytes)) return COCODIFF_ALIASING;
+    MoveParams p;
+    std::memset(&p, 0, sizeof p);
+    p.n_slots = S;
+    p.H = H;
+    p.src_tok = D;
+    p.src_head = COMPACT_STRIDE;
+    p.dst_tok = D;
+    p.dst_head = (long long)S * D;
+    p.map = MAP_SCATTER;
+    p.T = T;
+    p.idx = idx;
+    p.n_active = n_active;
+    p.job[p.njobs++] = MoveJob{x_compact, x_cache, nullptr};
+    CK(launch_move(p, D, (cudaStream_t)stream));
+    return COCODIFF_OK;
+}
+
+}  // extern "C"

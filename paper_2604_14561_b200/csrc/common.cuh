@@ -1,0 +1,65 @@
+// Shared declarations of the CUDA side of libcocodiff (sm_100a only).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cocodiff {
+
+// How an output token slot o maps to source and destination tokens.
+enum TokenMap : int {
+    MAP_FULL = 0,     // src token = dst token = o                      (full exchange)
+    MAP_GATHER = 1,   // src token = idx[o / T] * T + o % T, dst = o    (compaction)
+    MAP_SCATTER = 2   // src token = o, dst token = idx[o / T] * T + o % T  (reconstruction)
+};
+
+struct MoveJob {
+    const uint16_t *src;
+    uint16_t *dst;
+    const uint16_t *w;   // RMSNorm weight [D]; nullptr = plain move
+};
+
+// One launch moves up to three tensors (jobs) of identical geometry.  Strides
+// are in elements.  A stride given as COMPACT_STRIDE is n_active * T * D, read
+// on the device.
+constexpr long long COMPACT_STRIDE = -1;
+
+struct MoveParams {
+    MoveJob job[3];
+    int njobs;
+    int n_slots;            // token slots covered by the grid (capacity)
+    int H;
+    long long src_tok, src_head, dst_tok, dst_head;
+    const float *cs;        // [S][D/2][2] or nullptr
+    float eps;
+    const int32_t *idx;     // active units (MAP_GATHER / MAP_SCATTER)
+    const int32_t *n_active;
+    int T;
+    int map;
+};
+
+struct SelectParams {
+    const unsigned long long *metric;  // [n]
+    int n, n_groups, g, n_cached;
+    uint8_t *mask;
+    int32_t *idx;
+    int32_t *n_active;
+};
+
+struct MetricParams {
+    const uint4 *prev, *cur;
+    unsigned long long *acc;      // [n] accumulators in the workspace (zero on entry)
+    unsigned int *ticket;         // block ticket in the workspace (zero on entry)
+    unsigned long long *metric;   // [n] out
+    long long unit_vecs;          // 16-byte vectors per selection unit
+    int chunks_per_unit;
+    int chunk_vecs;
+    int n_units;
+    SelectParams sel;
+};
+
+cudaError_t launch_move(const MoveParams &p, int D, cudaStream_t stream);
+cudaError_t launch_rope_table(float *cs, const int32_t *pos, int S, int D, double theta, cudaStream_t stream);
+cudaError_t launch_select(const SelectParams &p, cudaStream_t stream);
+cudaError_t launch_metric_select(const MetricParams &p, cudaStream_t stream);
+
+}  // namespace cocodiff

@@ -1,0 +1,102 @@
+"""The C-ABI library: it loads without a GPU, exports every symbol the header
+declares, and rejects bad arguments before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2604_14561_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "cocodiff.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(cocodiff_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported_and_bound():
+    names = _declared()
+    assert len(names) >= 14
+    handle = ctypes.CDLL(binding.LIB_PATH)
+    for n in names:
+        assert hasattr(handle, n), n
+    assert set(names) == set(binding.SIGNATURES), set(names) ^ set(binding.SIGNATURES)
+
+
+def test_status_strings_and_version():
+    assert binding.version() >= 100
+    assert binding.status_string(0) == "ok"
+    for code in range(-6, 0):
+        assert binding.status_string(code) != "unknown status"
+
+
+A = 1 << 20          # fake, 16-byte aligned "device addresses"; never dereferenced:
+                     # every call below fails validation before any launch
+
+
+def _addr(i):
+    return A * (i + 1)
+
+
+def test_shape_validation():
+    q, k, v, qh, kh, vh = (_addr(i) * 64 for i in range(6))
+    ok = dict(P=2, S=8, H=4, D=64)
+    for bad, want in ((dict(P=3), -2), (dict(S=7), -2), (dict(H=3), -2), (dict(D=48), -2), (dict(D=8), -2),
+                      (dict(P=8, S=8, H=4), -2), (dict(P=0), -1), (dict(H=0), -1)):
+        a = dict(ok, **bad)
+        rc = binding.ulysses_a2a(q, k, v, qh, kh, vh, a["P"], a["S"], a["H"], a["D"], check=False)
+        assert rc == want, (bad, rc)
+    assert binding.ulysses_a2a(q, k, v, qh, kh, vh, 2, 8, 4, 64, order=7, check=False) == -1
+
+
+def test_pointer_validation():
+    q, k, v, qh, kh, vh = (_addr(i) * 64 for i in range(6))
+    assert binding.ulysses_a2a(q + 2, k, v, qh, kh, vh, 2, 8, 4, 64, check=False) == -3
+    assert binding.ulysses_a2a(q, None, v, qh, kh, vh, 2, 8, 4, 64, check=False) == -1      # half a pair
+    assert binding.ulysses_a2a(q, k, v, q + 16, kh, vh, 2, 8, 4, 64, check=False) == -6     # in/out overlap
+    assert binding.ulysses_a2a(q, k, v, qh, qh, vh, 2, 8, 4, 64, check=False) == -6         # out/out overlap
+    w, cs = _addr(40), _addr(41)
+    assert binding.prologue(q, k, v, qh, kh, vh, None, w, 1e-6, cs, 2, 8, 4, 64, check=False) == -1
+    assert binding.prologue(q, k, v, qh, kh, vh, w, w, -1.0, cs, 2, 8, 4, 64, check=False) == -1
+    assert binding.prologue(q, k, v, qh, kh, vh, w, w, 1e-6, cs + 4, 2, 8, 4, 64, check=False) == -3
+    # norm + rope in place is allowed to alias exactly, not partially
+    assert binding.qk_norm_rope(q, None, q + 32, None, w, None, 1e-6, cs, 8, 4, 64, check=False) == -6
+    assert binding.qk_norm_rope(q, None, None, None, w, None, 1e-6, cs, 8, 4, 64, check=False) == -1
+
+
+def test_vmajor_validation():
+    prev, cur, comp = (_addr(i) * 64 for i in range(3))
+    m, mask, idx, na, ws = (_addr(10 + i) for i in range(5))
+    need = binding.vmajor_workspace_bytes(2, 64, 4, 64, 8)
+    assert need >= 8 * 8 + 4 and need % 256 == 0
+    args = dict(P=2, S=64, H=4, D=64, T=8, r=0.5, n_groups=1)
+
+    def call(ws_bytes=need, **kw):
+        a = dict(args, **kw)
+        return binding.vmajor_select_compact(prev, cur, a["P"], a["S"], a["H"], a["D"], a["T"], a["r"],
+                                             a["n_groups"], m, mask, idx, na, comp, ws, ws_bytes, check=False)
+    assert call(T=3) == -2              # T must divide S/P
+    assert call(T=0) == -1
+    assert call(r=1.5) == -1 and call(r=-0.1) == -1 and call(r=float("nan")) == -1
+    assert call(n_groups=3) == -2 and call(n_groups=0) == -1
+    assert call(ws_bytes=need - 1) == -4
+    assert binding.vmajor_select(m, 10, 0.5, 3, mask, idx, na, check=False) == -2
+    assert binding.vmajor_select(m, 10, 2.0, 1, mask, idx, na, check=False) == -1
+    assert binding.pack_active(cur, None, 0.0, None, idx, na, cur, 2, 64, 4, 64, 8, check=False) == -6
+    assert binding.unpack(comp, idx, na, comp + 16, 2, 64, 4, 64, 8, check=False) == -6
+    assert binding.unpack(comp, None, na, cur, 2, 64, 4, 64, 8, check=False) == -1
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", binding.LIB_PATH + ".absent")
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        binding.lib()

@@ -1,0 +1,226 @@
+"""GPU parity of the V-Major path (metric, selection, compaction, unpack)
+against the CPU oracle through the C ABI: everything here is bit-exact except
+the normed and rotated values inside compacted Q/K (2 bf16 ulp)."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+import oracle
+from paper_2604_14561_b200 import binding, synth
+
+from gpu_util import Guarded, dev, rope_table, u16
+from helpers import assert_norm_rope_close
+
+
+class Selector:
+    """Device buffers of one V-Major call."""
+
+    def __init__(self, P, S, H, D, T):
+        self.shape = (P, S, H, D, T)
+        n = S // T
+        self.n = n
+        self.metric = torch.zeros(max(n, 1), dtype=torch.int64, device="cuda")
+        self.mask = torch.full((max(n, 1),), 77, dtype=torch.uint8, device="cuda")
+        self.idx = torch.full((max(n, 1),), -1, dtype=torch.int32, device="cuda")
+        self.n_active = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+        self.ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
+        self.ws = torch.full((self.ws_bytes,), 0xAB, dtype=torch.uint8, device="cuda")   # dirty on purpose
+        self.v_compact = Guarded(S * H * D)
+
+    def run(self, prev_v, cur_v, r, n_groups, compact=True, stream=None):
+        P, S, H, D, T = self.shape
+        binding.vmajor_select_compact(prev_v, cur_v, P, S, H, D, T, r, n_groups, self.metric, self.mask,
+                                      self.idx, self.n_active, self.v_compact.t if compact else None,
+                                      self.ws, self.ws_bytes, stream=stream)
+        torch.cuda.synchronize()
+        na = int(self.n_active.item())
+        return (self.metric.cpu().numpy().view(np.uint64)[:self.n], self.mask.cpu().numpy()[:self.n],
+                self.idx.cpu().numpy()[:na], na)
+
+
+def _pair(S, H, D, T, seed, frac=0.25):
+    rng = np.random.default_rng(seed)
+    prev = rng.normal(0, 1, (S, H, D)).astype(np.float32)
+    cur = prev + rng.normal(0, 1e-3, prev.shape).astype(np.float32)
+    n = S // T
+    hot = np.sort(rng.choice(n, max(1, int(frac * n)), replace=False))
+    for u in hot:
+        cur[u * T:(u + 1) * T] += rng.normal(0, 0.5, (T, H, D)).astype(np.float32)
+    return synth.f32_to_bf16_bits(prev), synth.f32_to_bf16_bits(cur), hot
+
+
+@pytest.mark.parametrize("P,S,H,D,T,n_groups", [
+    (2, 256, 4, 64, 16, 1), (2, 256, 4, 64, 16, 2), (4, 512, 4, 128, 1, 4), (4, 512, 4, 128, 1, 1),
+    (3, 96, 3, 32, 8, 12), (1, 40, 2, 256, 5, 1), (8, 2560, 8, 128, 64, 4), (2, 1200, 2, 64, 1, 1)])
+@pytest.mark.parametrize("r", [0.0, 0.3, 0.8, 1.0])
+def test_metric_selection_and_v_compaction(P, S, H, D, T, n_groups, r):
+    prev, cur, _ = _pair(S, H, D, T, seed=S + T)
+    sel = Selector(P, S, H, D, T)
+    metric, mask, idx, na = sel.run(dev(prev), dev(cur), r, n_groups)
+    m_ref = oracle.vmajor_metric(prev, cur, P, T)
+    assert np.array_equal(metric, m_ref)
+    mask_ref, idx_ref, na_ref = oracle.vmajor_select(m_ref, n_groups, r)
+    assert na == na_ref and np.array_equal(mask, mask_ref) and np.array_equal(idx, idx_ref)
+    comp_ref = oracle.pack_active(cur, idx_ref, P, T)
+    got = sel.v_compact.host()[:comp_ref.size].reshape(comp_ref.shape)
+    assert np.array_equal(got, comp_ref)
+    assert np.all(sel.v_compact.host()[comp_ref.size:] == 0x5A5A), "nothing beyond the compact extent is written"
+    sel.v_compact.assert_guards()
+    # a second call on the same (now used) workspace gives the same answer
+    metric2, mask2, idx2, na2 = sel.run(dev(prev), dev(cur), r, n_groups, compact=False)
+    assert np.array_equal(metric2, m_ref) and np.array_equal(mask2, mask_ref) and na2 == na_ref
+
+
+def test_metric_special_values():
+    S, H, D, T = 64, 2, 64, 4
+    prev = synth.f32_to_bf16_bits(np.zeros((S, H, D), np.float32))
+    cur = prev.copy()
+    cur[3, 1, 5] = 0x7FC0            # NaN
+    cur[20, 0, 0] = 0x7F7F           # largest finite bf16: saturates
+    cur[40, 1, 63] = 0x3880          # 2^-14 -> 4
+    cur[41, 1, 63] = 0x3700          # 2^-17 -> 0
+    sel = Selector(1, S, H, D, T)
+    metric, _, _, _ = sel.run(dev(prev), dev(cur), 0.5, 1, compact=False)
+    assert np.array_equal(metric, oracle.vmajor_metric(prev, cur, 1, T))
+    assert metric[0] == 2 ** 32 - 1 and metric[5] == 2 ** 32 - 1 and metric[10] == 4
+    same, _, _, na = sel.run(dev(cur), dev(cur), 0.5, 1, compact=False)
+    assert np.all(np.delete(same, 0) == 0)      # NaN - NaN is NaN: unit 0 stays saturated
+
+
+@pytest.mark.parametrize("n,n_groups", [(144, 1), (1000, 1), (1000, 8), (5000, 1), (21024, 1), (4096, 2), (513, 1), (600, 600)])
+def test_selection_alone_with_ties_and_wide_keys(n, n_groups):
+    rng = np.random.default_rng(n + n_groups)
+    for r, kind in ((0.8, "ties"), (0.5, "wide"), (0.999, "ties"), (0.0, "wide"), (1.0, "ties"), (0.25, "equal")):
+        if kind == "ties":
+            m = rng.integers(0, 7, n).astype(np.uint64)
+        elif kind == "equal":
+            m = np.full(n, 12345, np.uint64)
+        else:
+            m = rng.integers(0, 2 ** 63, n).astype(np.uint64) * np.uint64(2) + rng.integers(0, 2, n).astype(np.uint64)
+            m[rng.integers(0, n, n // 4)] = m[0]
+        mask = torch.full((n,), 9, dtype=torch.uint8, device="cuda")
+        idx = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        na = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+        binding.vmajor_select(dev(m), n, r, n_groups, mask, idx, na)
+        torch.cuda.synchronize()
+        mask_ref, idx_ref, na_ref = oracle.vmajor_select(m, n_groups, r)
+        assert int(na.item()) == na_ref, (r, kind)
+        assert np.array_equal(mask.cpu().numpy(), mask_ref), (r, kind)
+        assert np.array_equal(idx.cpu().numpy()[:na_ref], idx_ref), (r, kind)
+        assert np.all(idx.cpu().numpy()[na_ref:] == -1)
+
+
+@pytest.mark.parametrize("P,S,H,D,T", [(2, 256, 4, 64, 16), (4, 512, 4, 128, 1), (3, 99, 3, 32, 11), (2, 384, 2, 256, 64)])
+def test_pack_active_qk_and_unpack(P, S, H, D, T):
+    rng = np.random.default_rng(S)
+    n = S // T
+    x = synth.normal_bf16(5, "x", S * H * D).reshape(S, H, D)
+    w = synth.normal_bf16(5, "w", D, 1.0, 0.1)
+    pos = rng.integers(0, 150, (S, 2)).astype(np.int32)
+    cs_ref = oracle.rope_table_2d(pos, D, 10000.0)
+    cs = rope_table(pos, D, 10000.0)
+    normed, normed_f = oracle.norm_rope(x, w, 1e-6, cs_ref, want_f32=True)
+    for k in (0, 1, n // 3, n):
+        idx_np = np.sort(rng.choice(n, k, replace=False)).astype(np.int32)
+        idx = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        idx[:k] = dev(idx_np)
+        na = torch.tensor([k], dtype=torch.int32, device="cuda")
+        comp = Guarded(S * H * D)
+        binding.pack_active(dev(x), dev(w), 1e-6, cs, idx, na, comp.t, P, S, H, D, T)
+        torch.cuda.synchronize()
+        comp.assert_guards()
+        ref = oracle.pack_active(normed, idx_np, P, T)
+        tok = (idx_np[:, None] * T + np.arange(T)[None, :]).reshape(-1)
+        ref_f32 = np.ascontiguousarray(normed_f[tok].transpose(1, 0, 2))
+        got = comp.host()[:ref.size].reshape(ref.shape)
+        if k:
+            assert_norm_rope_close(got, ref, ref_f32, "compact q/k")
+        assert np.all(comp.host()[ref.size:] == 0x5A5A)
+        # plain move of the same units is bit-exact
+        plain = Guarded(S * H * D)
+        binding.pack_active(dev(x), None, 0.0, None, idx, na, plain.t, P, S, H, D, T)
+        torch.cuda.synchronize()
+        ref_plain = oracle.pack_active(x, idx_np, P, T)
+        assert np.array_equal(plain.host()[:ref_plain.size].reshape(ref_plain.shape), ref_plain)
+        # scatter over a cached tensor
+        old = synth.normal_bf16(6, "old", S * H * D).reshape(H, S, D)
+        cache = Guarded(S * H * D, fill=old)
+        binding.unpack(plain.t, idx, na, cache.t, P, S, H, D, T)
+        torch.cuda.synchronize()
+        cache.assert_guards()
+        want = oracle.unpack(ref_plain, idx_np, old.copy(), P, T)
+        assert np.array_equal(cache.host((H, S, D)), want)
+        binding.unpack(plain.t, idx, na, cache.t, P, S, H, D, T)          # idempotent
+        torch.cuda.synchronize()
+        assert np.array_equal(cache.host((H, S, D)), want)
+
+
+def _temporal_cfg(small):
+    cfg = synth.config("temporal")
+    if small:
+        cfg.update(grid=(32, 24), P=4, H=4, D=64, T=16, steps=4)
+        cfg["S"] = 32 * 24
+    return cfg
+
+
+@pytest.mark.parametrize("small", [True, False], ids=["reduced", "full-size"])
+def test_temporal_steps_select_compact_unpack(small):
+    """Several denoising steps: step 0 runs the full prologue and fills the
+    caches; every later step selects on V, compacts V, K, Q (norm + RoPE fused)
+    and scatters them over the caches.  Compared with the oracle step by step;
+    the active set must equal the generator's strongly perturbed tiles."""
+    cfg = _temporal_cfg(small)
+    P, S, H, D, T = cfg["P"], cfg["S"], cfg["H"], cfg["D"], cfg["T"]
+    E, n = S * H * D, S // T
+    seq = synth.TemporalSequence(cfg)
+    cs_ref = oracle.rope_table_2d(seq.pos, D, cfg["theta"])
+    cs = rope_table(seq.pos, D, cfg["theta"])
+    wq, wk = dev(seq.wq), dev(seq.wk)
+    cur = seq.current()
+    # step 0: full exchange on both sides
+    cache_ref = dict(zip("qkv", oracle.prologue(cur["q"], cur["k"], cur["v"], seq.wq, seq.wk, cfg["eps"], cs_ref, P)))
+    cache = {x: Guarded(E) for x in "qkv"}
+    d = {x: dev(cur[x]) for x in "qkv"}
+    binding.prologue(d["q"], d["k"], d["v"], cache["q"].t, cache["k"].t, cache["v"].t, wq, wk, cfg["eps"], cs,
+                     P, S, H, D, order=binding.V_FIRST, stream_qk=None, stream_v=torch.cuda.Stream())
+    torch.cuda.synchronize()
+    assert np.array_equal(cache["v"].host((H, S, D)), cache_ref["v"])
+    # Q and K caches start from the oracle's bits on both sides so that later steps compare exactly
+    for x in "qk":
+        cache[x].t.copy_(dev(cache_ref[x]).reshape(-1))
+    prev_v = cur["v"]
+    sel = Selector(P, S, H, D, T)
+    comp = {x: Guarded(E) for x in "qk"}
+    for step in range(1, cfg["steps"]):
+        hot = seq.advance()
+        cur = seq.current()
+        d = {x: dev(cur[x]) for x in "qkv"}
+        metric, mask, idx, na = sel.run(dev(prev_v), d["v"], cfg["r"], cfg["n_groups"])
+        m_ref = oracle.vmajor_metric(prev_v, cur["v"], P, T)
+        mask_ref, idx_ref, na_ref = oracle.vmajor_select(m_ref, cfg["n_groups"], cfg["r"])
+        assert np.array_equal(metric, m_ref) and np.array_equal(mask, mask_ref)
+        assert na == na_ref and np.array_equal(idx, idx_ref)
+        assert np.array_equal(idx, hot), "active set = the strongly perturbed tiles"
+        for x, w, w_np in (("k", wk, seq.wk), ("q", wq, seq.wq)):
+            binding.pack_active(d[x], w, cfg["eps"], cs, sel.idx, sel.n_active, comp[x].t, P, S, H, D, T)
+        for x, src in (("v", sel.v_compact), ("k", comp["k"]), ("q", comp["q"])):
+            binding.unpack(src.t, sel.idx, sel.n_active, cache[x].t, P, S, H, D, T)
+        torch.cuda.synchronize()
+        # oracle: norm + RoPE on all rows, extract the active ones, scatter
+        oracle.unpack(oracle.pack_active(cur["v"], idx_ref, P, T), idx_ref, cache_ref["v"], P, T)
+        assert np.array_equal(cache["v"].host((H, S, D)), cache_ref["v"]), f"V cache, step {step}"
+        tok = (idx_ref[:, None] * T + np.arange(T)[None, :]).reshape(-1)
+        for x, w_np in (("k", seq.wk), ("q", seq.wq)):
+            ref, ref_f = oracle.norm_rope(cur[x], w_np, cfg["eps"], cs_ref, want_f32=True)
+            oracle.unpack(oracle.pack_active(ref, idx_ref, P, T), idx_ref, cache_ref[x], P, T)
+            got = cache[x].host((H, S, D))
+            inactive = np.ones(S, bool)
+            inactive[tok] = False
+            assert np.array_equal(got[:, inactive], cache_ref[x][:, inactive]), f"{x}: cached rows must not move"
+            assert_norm_rope_close(got[:, tok], cache_ref[x][:, tok],
+                                   np.ascontiguousarray(ref_f[tok].transpose(1, 0, 2)), f"{x} cache, step {step}")
+            cache[x].t.copy_(dev(cache_ref[x]).reshape(-1))     # re-align the two sides bit for bit
+            cache[x].assert_guards()
+        prev_v = cur["v"]
