@@ -250,6 +250,11 @@ def run_ours(args):
     value = aggregate_gbs(step_bytes, world, ms_per_step)
 
     line = None
+    if rank == 0 and args.only_main:
+        print(json.dumps({"metric": METRIC, "value": value, "unit": "GB/s", "us_per_layer": 1e3 * ms_per_step,
+                          "n_gpus": world, "steps": args.steps, "note": "--only-main: headline loop only",
+                          "clocks": clocks}, ensure_ascii=False))
+        return
     if rank == 0:
         # ---- per-order detail, per-step events (this GPU only) --------------
         orders = {}
@@ -406,6 +411,8 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--only-main", action="store_true",
+                    help="run only the headline loop (short launch list for profiling)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
