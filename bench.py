@@ -251,11 +251,9 @@ def run_ours(args):
 
     line = None
     if rank == 0 and args.only_main:
-        print(json.dumps({"metric": METRIC, "value": value, "unit": "GB/s", "us_per_layer": 1e3 * ms_per_step,
-                          "n_gpus": world, "steps": args.steps, "note": "--only-main: headline loop only",
-                          "clocks": clocks}, ensure_ascii=False))
-        return
-    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": "GB/s", "us_per_layer": 1e3 * ms_per_step,
+                "n_gpus": world, "steps": args.steps, "note": "--only-main: headline loop only", "clocks": clocks}
+    elif rank == 0:
         # ---- per-order detail, per-step events (this GPU only) --------------
         orders = {}
         for name, order in (("v_first", binding.V_FIRST), ("lump", binding.LUMP)):
