@@ -357,15 +357,16 @@ def other_configs(torch, binding, args):
         binding.rope_table_2d(cs, dev(L["pos"], torch), S, D, cfg["theta"])
         qh, kh, vh = (torch.empty(E, dtype=torch.int16, device="cuda") for _ in range(3))
 
-        def full():
+        def full(order):
             binding.prologue(q, k, v, qh, kh, vh, wq, wk, cfg["eps"], cs, P, S, H, D,
-                             order=binding.V_FIRST, stream_qk=sq, stream_v=sv)
-        cold = time_steps(torch, full, sq, iters, 3, flush=flush)
-        warm = time_steps(torch, full, sq, iters, 3)
+                             order=order, stream_qk=sq, stream_v=sv)
         b = algorithmic_bytes(cfg)
-        out[name] = {"bytes": b, "us_cold_l2": 1e3 * statistics.median(cold),
-                     "gbs_cold_l2": b / (statistics.median(cold) * 1e-3) / 1e9,
-                     "us_warm_l2": 1e3 * statistics.median(warm)}
+        out[name] = {"bytes": b}
+        for oname, order in (("v_first", binding.V_FIRST), ("lump", binding.LUMP)):
+            cold = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 3, flush=flush))
+            warm = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 3))
+            out[name][oname] = {"us_cold_l2": 1e3 * cold, "gbs_cold_l2": b / (cold * 1e-3) / 1e9,
+                                "us_warm_l2": 1e3 * warm}
         if name != "temporal":
             continue
         # selective step: metric + selection + V compaction, K/Q compaction (norm + RoPE fused), three scatters
@@ -384,22 +385,22 @@ def other_configs(torch, binding, args):
         na = torch.zeros(1, dtype=torch.int32, device="cuda")
         comp = [torch.empty(E, dtype=torch.int16, device="cuda") for _ in range(3)]
 
-        def selective():
-            binding.vmajor_select_compact(v, cur_v, P, S, H, D, T, r, n_groups, metric, mask, idx, na, comp[2],
-                                          ws, ws_bytes, stream=sq)
-            binding.pack_active(k, wk, cfg["eps"], cs, idx, na, comp[1], P, S, H, D, T, stream=sq)
-            binding.pack_active(q, wq, cfg["eps"], cs, idx, na, comp[0], P, S, H, D, T, stream=sq)
-            binding.unpack(comp[2], idx, na, vh, P, S, H, D, T, stream=sq)
-            binding.unpack(comp[1], idx, na, kh, P, S, H, D, T, stream=sq)
-            binding.unpack(comp[0], idx, na, qh, P, S, H, D, T, stream=sq)
-        cold = time_steps(torch, selective, sq, iters, 3, flush=flush)
+        def selective(order):
+            binding.selective_prologue(v, q, k, cur_v, wq, wk, cfg["eps"], cs, P, S, H, D, T, r, n_groups,
+                                       metric, mask, idx, na, comp[0], comp[1], comp[2], qh, kh, vh,
+                                       ws, ws_bytes, order=order, stream_qk=sq, stream_v=sv)
+        sel = {}
+        for oname, order in (("lump", binding.LUMP), ("v_first", binding.V_FIRST)):
+            cold = time_steps(torch, lambda: selective(order), sq, iters, 3, flush=flush)
+            sel[oname] = 1e3 * statistics.median(cold)
         n_act = int(na.item())
         tile = T * H * D * 2
         sb = 2 * E * 2 + 3 * 2 * n_act * tile + 3 * 2 * n_act * tile
+        best = min(sel.values())
         out["temporal_selective_step"] = {"n_active": n_act, "n_units": n, "bytes": sb,
-                                          "us_cold_l2": 1e3 * statistics.median(cold),
-                                          "gbs_cold_l2": sb / (statistics.median(cold) * 1e-3) / 1e9,
-                                          "launches_per_step": 8}
+                                          "us_cold_l2": sel, "gbs_cold_l2_best": sb / (best * 1e-6) / 1e9,
+                                          "launches_per_step": {"lump": 4, "v_first": 5},
+                                          "api": "cocodiff_selective_prologue"}
     return out
 
 

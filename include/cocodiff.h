@@ -156,11 +156,43 @@ int cocodiff_pack_active(const uint16_t *x, const uint16_t *w, float eps, const 
                          const int32_t *idx, const int32_t *n_active, uint16_t *x_compact,
                          int P, int S, int H, int D, int T, void *stream);
 
+/* The same extraction for Q, K and V in one launch (Q, K normalised and rotated,
+ * V moved); any (x, x_compact) pair may be NULL/NULL. */
+int cocodiff_pack_active_qkv(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                             const uint16_t *wq, const uint16_t *wk, float eps, const float *cs,
+                             const int32_t *idx, const int32_t *n_active,
+                             uint16_t *q_compact, uint16_t *k_compact, uint16_t *v_compact,
+                             int P, int S, int H, int D, int T, void *stream);
+
 /* Receiver-side reconstruction (Section III-D, "Post-Phase 2"): indexed scatter
  * x_cache[h][idx[a]*T + j][:] = x_compact[h][a][j][:]; all other rows of the
  * cached HEAD tensor keep their bits. */
 int cocodiff_unpack(const uint16_t *x_compact, const int32_t *idx, const int32_t *n_active,
                     uint16_t *x_cache, int P, int S, int H, int D, int T, void *stream);
+
+/* The same scatter for Q, K and V in one launch; any pair may be NULL/NULL. */
+int cocodiff_unpack_qkv(const uint16_t *q_compact, const uint16_t *k_compact, const uint16_t *v_compact,
+                        const int32_t *idx, const int32_t *n_active,
+                        uint16_t *q_cache, uint16_t *k_cache, uint16_t *v_cache,
+                        int P, int S, int H, int D, int T, void *stream);
+
+/* One selective step of a layer (Section III-D; timeline of Figure 4(d)):
+ * metric and selection on V, compaction of the active units of V (moved) and of
+ * Q, K (normalised and rotated on the way), then - if the three caches are
+ * given - the scatter over the cached HEAD tensors.  V_FIRST with two streams:
+ * metric, selection and V's compaction run on stream_v, Q and K start on
+ * stream_qk as soon as the index list exists; LUMP or equal streams: one stream,
+ * the three compactions in one launch.  Stream semantics as for
+ * cocodiff_ulysses_a2a; outputs and workspace as for
+ * cocodiff_vmajor_select_compact.  The caches are all given or all NULL. */
+int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                                const uint16_t *wq, const uint16_t *wk, float eps, const float *cs,
+                                int P, int S, int H, int D, int T, double r, int n_groups,
+                                uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
+                                uint16_t *q_compact, uint16_t *k_compact, uint16_t *v_compact,
+                                uint16_t *q_cache, uint16_t *k_cache, uint16_t *v_cache,
+                                void *workspace, size_t workspace_bytes, cocodiff_order order,
+                                void *stream_qk, void *stream_v);
 
 #ifdef __cplusplus
 }

@@ -39,6 +39,9 @@ SIGNATURES = {
     "cocodiff_vmajor_select": (_I, [_P, _I, _D, _I, _P, _P, _P, _P]),
     "cocodiff_pack_active": (_I, [_P, _P, _F, _P, _P, _P, _P] + [_I] * 5 + [_P]),
     "cocodiff_unpack": (_I, [_P, _P, _P, _P] + [_I] * 5 + [_P]),
+    "cocodiff_pack_active_qkv": (_I, [_P] * 5 + [_F] + [_P] * 6 + [_I] * 5 + [_P]),
+    "cocodiff_unpack_qkv": (_I, [_P] * 8 + [_I] * 5 + [_P]),
+    "cocodiff_selective_prologue": (_I, [_P] * 6 + [_F, _P] + [_I] * 5 + [_D, _I] + [_P] * 11 + [_Z, _I, _P, _P]),
 }
 
 
@@ -159,3 +162,27 @@ def pack_active(x, w, eps, cs, idx, n_active, x_compact, P, S, H, D, T, stream=N
 def unpack(x_compact, idx, n_active, x_cache, P, S, H, D, T, stream=None, check=True):
     return _call("cocodiff_unpack", _ptr(x_compact), _ptr(idx), _ptr(n_active), _ptr(x_cache),
                  P, S, H, D, T, _stream(stream), check=check)
+
+
+def pack_active_qkv(q, k, v, wq, wk, eps, cs, idx, n_active, q_compact, k_compact, v_compact,
+                    P, S, H, D, T, stream=None, check=True):
+    return _call("cocodiff_pack_active_qkv", _ptr(q), _ptr(k), _ptr(v), _ptr(wq), _ptr(wk), eps, _ptr(cs),
+                 _ptr(idx), _ptr(n_active), _ptr(q_compact), _ptr(k_compact), _ptr(v_compact),
+                 P, S, H, D, T, _stream(stream), check=check)
+
+
+def unpack_qkv(q_compact, k_compact, v_compact, idx, n_active, q_cache, k_cache, v_cache,
+               P, S, H, D, T, stream=None, check=True):
+    return _call("cocodiff_unpack_qkv", _ptr(q_compact), _ptr(k_compact), _ptr(v_compact), _ptr(idx),
+                 _ptr(n_active), _ptr(q_cache), _ptr(k_cache), _ptr(v_cache), P, S, H, D, T,
+                 _stream(stream), check=check)
+
+
+def selective_prologue(prev_v, q, k, v, wq, wk, eps, cs, P, S, H, D, T, r, n_groups, metric, mask, idx,
+                       n_active, q_compact, k_compact, v_compact, q_cache, k_cache, v_cache,
+                       workspace, workspace_bytes, order=V_FIRST, stream_qk=None, stream_v=None, check=True):
+    return _call("cocodiff_selective_prologue", _ptr(prev_v), _ptr(q), _ptr(k), _ptr(v), _ptr(wq), _ptr(wk),
+                 eps, _ptr(cs), P, S, H, D, T, r, n_groups, _ptr(metric), _ptr(mask), _ptr(idx),
+                 _ptr(n_active), _ptr(q_compact), _ptr(k_compact), _ptr(v_compact), _ptr(q_cache),
+                 _ptr(k_cache), _ptr(v_cache), _ptr(workspace), workspace_bytes, order,
+                 _stream(stream_qk), _stream(stream_v), check=check)

@@ -130,6 +130,118 @@ int check_pairs(const uint16_t *const in[3], uint16_t *const out[3], size_t byte
     return COCODIFF_OK;
 }
 
+
+// ---- V-Major helpers --------------------------------------------------------
+size_t vmajor_ws_bytes(int S, int T) {
+    const size_t n = (size_t)(S / T);
+    return ((n * 8 + 255) / 256) * 256 + 256;  // accumulators, then the ticket
+}
+
+int check_select(const uint16_t *prev_v, const uint16_t *cur_v, int P, int S, int H, int D, int T, double r,
+                 int n_groups, const uint64_t *metric, const uint8_t *mask, const int32_t *idx,
+                 const int32_t *n_active, const void *workspace, size_t workspace_bytes) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    rc = check_unit(P, S, T);
+    if (rc) return rc;
+    if (!prev_v || !cur_v || !metric || !mask || !idx || !n_active || !workspace || n_groups < 1 ||
+        !(r >= 0.0 && r <= 1.0))
+        return COCODIFF_INVALID_ARG;
+    if ((S / T) % n_groups != 0) return COCODIFF_BAD_SHAPE;
+    if (!aligned16(prev_v) || !aligned16(cur_v) || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        (reinterpret_cast<uintptr_t>(metric) & 7u) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
+        (reinterpret_cast<uintptr_t>(n_active) & 3u))
+        return COCODIFF_MISALIGNED;
+    if (workspace_bytes < vmajor_ws_bytes(S, T)) return COCODIFF_WORKSPACE_TOO_SMALL;
+    return COCODIFF_OK;
+}
+
+// in/out pairs of a compaction or scatter: both or neither, aligned, disjoint.
+int check_tiles(const uint16_t *const in[3], uint16_t *const out[3], int S, int H, int D, const int32_t *idx,
+                const int32_t *n_active) {
+    if (!idx || !n_active) return COCODIFF_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(n_active) & 3u))
+        return COCODIFF_MISALIGNED;
+    return check_pairs(in, out, (size_t)S * H * D * 2);
+}
+
+int enqueue_metric_select(const uint16_t *prev_v, const uint16_t *cur_v, int S, int H, int D, int T, double r,
+                          int n_groups, uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
+                          void *workspace, cudaStream_t st) {
+    const int n = S / T;
+    const size_t need = vmajor_ws_bytes(S, T);
+    MetricParams mp;
+    std::memset(&mp, 0, sizeof mp);
+    mp.prev = reinterpret_cast<const uint4 *>(prev_v);
+    mp.cur = reinterpret_cast<const uint4 *>(cur_v);
+    mp.acc = reinterpret_cast<unsigned long long *>(workspace);
+    mp.ticket = reinterpret_cast<unsigned int *>(reinterpret_cast<char *>(workspace) + (need - 256));
+    mp.metric = reinterpret_cast<unsigned long long *>(metric);
+    mp.unit_vecs = (long long)T * H * D / 8;
+    mp.chunk_vecs = 512;
+    mp.chunks_per_unit = (int)((mp.unit_vecs + mp.chunk_vecs - 1) / mp.chunk_vecs);
+    mp.n_units = n;
+    mp.sel.metric = mp.metric;
+    mp.sel.n = n;
+    mp.sel.n_groups = n_groups;
+    mp.sel.g = n / n_groups;
+    mp.sel.n_cached = (int)std::floor(r * (double)mp.sel.g);
+    mp.sel.mask = mask;
+    mp.sel.idx = idx;
+    mp.sel.n_active = n_active;
+    CK(cudaMemsetAsync(workspace, 0, need, st));
+    CK(launch_metric_select(mp, st));
+    return COCODIFF_OK;
+}
+
+// Compaction of up to three tensors in one launch; slot order (Q, K, V), V's blocks first.
+int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint16_t *wq, const uint16_t *wk,
+                 float eps, const float *cs, const int32_t *idx, const int32_t *n_active, int slots, int S,
+                 int H, int D, int T, cudaStream_t st) {
+    (void)S;
+    MoveParams p;
+    std::memset(&p, 0, sizeof p);
+    p.n_slots = slots;
+    p.H = H;
+    p.src_tok = (long long)H * D;
+    p.src_head = D;
+    p.dst_tok = D;
+    p.dst_head = COMPACT_STRIDE;
+    p.map = MAP_GATHER;
+    p.T = T;
+    p.idx = idx;
+    p.n_active = n_active;
+    p.cs = cs;
+    p.eps = eps;
+    if (in[2]) p.job[p.njobs++] = MoveJob{in[2], out[2], nullptr};
+    if (in[0]) p.job[p.njobs++] = MoveJob{in[0], out[0], wq};
+    if (in[1]) p.job[p.njobs++] = MoveJob{in[1], out[1], wk};
+    if (p.njobs == 0) return COCODIFF_OK;
+    CK(launch_move(p, D, st));
+    return COCODIFF_OK;
+}
+
+int enqueue_unpack(const uint16_t *const in[3], uint16_t *const out[3], const int32_t *idx,
+                   const int32_t *n_active, int slots, int S, int H, int D, int T, cudaStream_t st) {
+    MoveParams p;
+    std::memset(&p, 0, sizeof p);
+    p.n_slots = slots;
+    p.H = H;
+    p.src_tok = D;
+    p.src_head = COMPACT_STRIDE;
+    p.dst_tok = D;
+    p.dst_head = (long long)S * D;
+    p.map = MAP_SCATTER;
+    p.T = T;
+    p.idx = idx;
+    p.n_active = n_active;
+    for (int i = 2; i >= 0; --i)
+        if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr};
+    if (p.njobs == 0) return COCODIFF_OK;
+    CK(launch_move(p, D, st));
+    return COCODIFF_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -302,8 +414,7 @@ size_t cocodiff_vmajor_workspace_bytes(int P, int S, int H, int D, int T) {
     (void)H;
     (void)D;
     if (P < 1 || T < 1 || S < 0) return 0;
-    const size_t n = (size_t)(S / T);
-    return ((n * 8 + 255) / 256) * 256 + 256;  // accumulators, then the ticket
+    return vmajor_ws_bytes(S, T);
 }
 
 int cocodiff_vmajor_select(const uint64_t *metric, int n, double r, int n_groups, uint8_t *mask,
@@ -331,49 +442,20 @@ int cocodiff_vmajor_select_compact(const uint16_t *prev_v, const uint16_t *cur_v
                                    int D, int T, double r, int n_groups, uint64_t *metric, uint8_t *mask,
                                    int32_t *idx, int32_t *n_active, uint16_t *v_compact, void *workspace,
                                    size_t workspace_bytes, void *stream) {
-    int rc = check_shape(P, S, H, D);
+    int rc = check_select(prev_v, cur_v, P, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace,
+                          workspace_bytes);
     if (rc) return rc;
-    rc = check_unit(P, S, T);
-    if (rc) return rc;
-    if (!prev_v || !cur_v || !metric || !mask || !idx || !n_active || !workspace || n_groups < 1 ||
-        !(r >= 0.0 && r <= 1.0))
-        return COCODIFF_INVALID_ARG;
-    const int n = S / T;
-    if (n % n_groups != 0) return COCODIFF_BAD_SHAPE;
-    if (!aligned16(prev_v) || !aligned16(cur_v) || !aligned16(v_compact) ||
-        (reinterpret_cast<uintptr_t>(workspace) & 255u) || (reinterpret_cast<uintptr_t>(metric) & 7u) ||
-        (reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(n_active) & 3u))
-        return COCODIFF_MISALIGNED;
-    const size_t need = cocodiff_vmajor_workspace_bytes(P, S, H, D, T);
-    if (workspace_bytes < need) return COCODIFF_WORKSPACE_TOO_SMALL;
-    const size_t bytes = (size_t)S * H * D * 2;
-    if (overlap(cur_v, bytes, v_compact, bytes) || overlap(prev_v, bytes, v_compact, bytes))
-        return COCODIFF_ALIASING;
+    const uint16_t *in[3] = {nullptr, nullptr, cur_v};
+    uint16_t *out[3] = {nullptr, nullptr, v_compact};
+    if (v_compact) {
+        rc = check_tiles(in, out, S, H, D, idx, n_active);
+        if (rc) return rc;
+        if (overlap(prev_v, (size_t)S * H * D * 2, v_compact, (size_t)S * H * D * 2)) return COCODIFF_ALIASING;
+    }
     cudaStream_t st = (cudaStream_t)stream;
-
-    MetricParams mp;
-    std::memset(&mp, 0, sizeof mp);
-    mp.prev = reinterpret_cast<const uint4 *>(prev_v);
-    mp.cur = reinterpret_cast<const uint4 *>(cur_v);
-    mp.acc = reinterpret_cast<unsigned long long *>(workspace);
-    mp.ticket = reinterpret_cast<unsigned int *>(reinterpret_cast<char *>(workspace) + (need - 256));
-    mp.metric = reinterpret_cast<unsigned long long *>(metric);
-    mp.unit_vecs = (long long)T * H * D / 8;
-    mp.chunk_vecs = 512;
-    mp.chunks_per_unit = (int)((mp.unit_vecs + mp.chunk_vecs - 1) / mp.chunk_vecs);
-    mp.n_units = n;
-    mp.sel.metric = mp.metric;
-    mp.sel.n = n;
-    mp.sel.n_groups = n_groups;
-    mp.sel.g = n / n_groups;
-    mp.sel.n_cached = (int)std::floor(r * (double)mp.sel.g);
-    mp.sel.mask = mask;
-    mp.sel.idx = idx;
-    mp.sel.n_active = n_active;
-    CK(cudaMemsetAsync(workspace, 0, need, st));
-    CK(launch_metric_select(mp, st));
-    if (v_compact)
-        return cocodiff_pack_active(cur_v, nullptr, 0.f, nullptr, idx, n_active, v_compact, P, S, H, D, T, stream);
+    rc = enqueue_metric_select(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, st);
+    if (rc) return rc;
+    if (v_compact) return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, S, S, H, D, T, st);
     return COCODIFF_OK;
 }
 
@@ -384,29 +466,31 @@ int cocodiff_pack_active(const uint16_t *x, const uint16_t *w, float eps, const 
     if (rc) return rc;
     rc = check_unit(P, S, T);
     if (rc) return rc;
-    if (!x || !idx || !n_active || !x_compact || !(eps >= 0.f)) return COCODIFF_INVALID_ARG;
-    if (!aligned16(x) || !aligned16(x_compact) || !aligned16(w) || !aligned16(cs) ||
-        (reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(n_active) & 3u))
-        return COCODIFF_MISALIGNED;
-    const size_t bytes = (size_t)S * H * D * 2;
-    if (overlap(x, bytes, x_compact, bytes)) return COCODIFF_ALIASING;
-    MoveParams p;
-    std::memset(&p, 0, sizeof p);
-    p.n_slots = S;
-    p.H = H;
-    p.src_tok = (long long)H * D;
-    p.src_head = D;
-    p.dst_tok = D;
-    p.dst_head = COMPACT_STRIDE;
-    p.map = MAP_GATHER;
-    p.T = T;
-    p.idx = idx;
-    p.n_active = n_active;
-    p.cs = w ? cs : nullptr;
-    p.eps = eps;
-    p.job[p.njobs++] = MoveJob{x, x_compact, w};
-    CK(launch_move(p, D, (cudaStream_t)stream));
-    return COCODIFF_OK;
+    if (!x || !x_compact || !(eps >= 0.f)) return COCODIFF_INVALID_ARG;
+    if (!aligned16(w) || !aligned16(cs)) return COCODIFF_MISALIGNED;
+    // one tensor: it travels in the Q slot when it is normalised, in the V slot otherwise
+    const uint16_t *in[3] = {w ? x : nullptr, nullptr, w ? nullptr : x};
+    uint16_t *out[3] = {w ? x_compact : nullptr, nullptr, w ? nullptr : x_compact};
+    rc = check_tiles(in, out, S, H, D, idx, n_active);
+    if (rc) return rc;
+    return enqueue_pack(in, out, w, nullptr, eps, cs, idx, n_active, S, S, H, D, T, (cudaStream_t)stream);
+}
+
+int cocodiff_pack_active_qkv(const uint16_t *q, const uint16_t *k, const uint16_t *v, const uint16_t *wq,
+                             const uint16_t *wk, float eps, const float *cs, const int32_t *idx,
+                             const int32_t *n_active, uint16_t *q_compact, uint16_t *k_compact,
+                             uint16_t *v_compact, int P, int S, int H, int D, int T, void *stream) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    rc = check_unit(P, S, T);
+    if (rc) return rc;
+    if ((q && !wq) || (k && !wk) || !(eps >= 0.f)) return COCODIFF_INVALID_ARG;
+    if (!aligned16(wq) || !aligned16(wk) || !aligned16(cs)) return COCODIFF_MISALIGNED;
+    const uint16_t *in[3] = {q, k, v};
+    uint16_t *out[3] = {q_compact, k_compact, v_compact};
+    rc = check_tiles(in, out, S, H, D, idx, n_active);
+    if (rc) return rc;
+    return enqueue_pack(in, out, wq, wk, eps, cs, idx, n_active, S, S, H, D, T, (cudaStream_t)stream);
 }
 
 int cocodiff_unpack(const uint16_t *x_compact, const int32_t *idx, const int32_t *n_active,
@@ -415,26 +499,94 @@ int cocodiff_unpack(const uint16_t *x_compact, const int32_t *idx, const int32_t
     if (rc) return rc;
     rc = check_unit(P, S, T);
     if (rc) return rc;
-    if (!x_compact || !idx || !n_active || !x_cache) return COCODIFF_INVALID_ARG;
-    if (!aligned16(x_compact) || !aligned16(x_cache) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
-        (reinterpret_cast<uintptr_t>(n_active) & 3u))
-        return COCODIFF_MISALIGNED;
+    if (!x_compact || !x_cache) return COCODIFF_INVALID_ARG;
+    const uint16_t *in[3] = {nullptr, nullptr, x_compact};
+    uint16_t *out[3] = {nullptr, nullptr, x_cache};
+    rc = check_tiles(in, out, S, H, D, idx, n_active);
+    if (rc) return rc;
+    return enqueue_unpack(in, out, idx, n_active, S, S, H, D, T, (cudaStream_t)stream);
+}
+
+int cocodiff_unpack_qkv(const uint16_t *q_compact, const uint16_t *k_compact, const uint16_t *v_compact,
+                        const int32_t *idx, const int32_t *n_active, uint16_t *q_cache, uint16_t *k_cache,
+                        uint16_t *v_cache, int P, int S, int H, int D, int T, void *stream) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    rc = check_unit(P, S, T);
+    if (rc) return rc;
+    const uint16_t *in[3] = {q_compact, k_compact, v_compact};
+    uint16_t *out[3] = {q_cache, k_cache, v_cache};
+    rc = check_tiles(in, out, S, H, D, idx, n_active);
+    if (rc) return rc;
+    return enqueue_unpack(in, out, idx, n_active, S, S, H, D, T, (cudaStream_t)stream);
+}
+
+int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const uint16_t *k,
+                                const uint16_t *v, const uint16_t *wq, const uint16_t *wk, float eps,
+                                const float *cs, int P, int S, int H, int D, int T, double r, int n_groups,
+                                uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
+                                uint16_t *q_compact, uint16_t *k_compact, uint16_t *v_compact,
+                                uint16_t *q_cache, uint16_t *k_cache, uint16_t *v_cache, void *workspace,
+                                size_t workspace_bytes, cocodiff_order order, void *stream_qk, void *stream_v) {
+    int rc = check_select(prev_v, v, P, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace,
+                          workspace_bytes);
+    if (rc) return rc;
+    if (order != COCODIFF_LUMP && order != COCODIFF_V_FIRST) return COCODIFF_INVALID_ARG;
+    if (!q || !k || !wq || !wk || !cs || !q_compact || !k_compact || !v_compact || !(eps >= 0.f))
+        return COCODIFF_INVALID_ARG;
+    if (!aligned16(wq) || !aligned16(wk) || !aligned16(cs)) return COCODIFF_MISALIGNED;
+    const bool do_unpack = q_cache || k_cache || v_cache;
+    if (do_unpack && !(q_cache && k_cache && v_cache)) return COCODIFF_INVALID_ARG;
+    const uint16_t *in[3] = {q, k, v};
+    uint16_t *comp[3] = {q_compact, k_compact, v_compact};
+    rc = check_tiles(in, comp, S, H, D, idx, n_active);
+    if (rc) return rc;
     const size_t bytes = (size_t)S * H * D * 2;
-    if (overlap(x_compact, bytes, x_cache, bytes)) return COCODIFF_ALIASING;
-    MoveParams p;
-    std::memset(&p, 0, sizeof p);
-    p.n_slots = S;
-    p.H = H;
-    p.src_tok = D;
-    p.src_head = COMPACT_STRIDE;
-    p.dst_tok = D;
-    p.dst_head = (long long)S * D;
-    p.map = MAP_SCATTER;
-    p.T = T;
-    p.idx = idx;
-    p.n_active = n_active;
-    p.job[p.njobs++] = MoveJob{x_compact, x_cache, nullptr};
-    CK(launch_move(p, D, (cudaStream_t)stream));
+    for (int i = 0; i < 3; ++i)
+        if (overlap(prev_v, bytes, comp[i], bytes)) return COCODIFF_ALIASING;
+    const uint16_t *comp_in[3] = {q_compact, k_compact, v_compact};
+    uint16_t *cache[3] = {q_cache, k_cache, v_cache};
+    if (do_unpack) {
+        rc = check_tiles(comp_in, cache, S, H, D, idx, n_active);
+        if (rc) return rc;
+        for (int i = 0; i < 3; ++i)
+            for (int j = 0; j < 3; ++j)
+                if (overlap(in[i], bytes, cache[j], bytes) || overlap(prev_v, bytes, cache[j], bytes))
+                    return COCODIFF_ALIASING;
+    }
+    // the host knows how many units will be active: grids are sized exactly
+    const int n = S / T, g = n / n_groups;
+    const int slots = (n - n_groups * (int)std::floor(r * (double)g)) * T;
+    cudaStream_t sq = (cudaStream_t)stream_qk, sv = (cudaStream_t)stream_v;
+    if (order == COCODIFF_LUMP || sv == sq) {
+        rc = enqueue_metric_select(prev_v, v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, sq);
+        if (rc) return rc;
+        rc = enqueue_pack(in, comp, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T, sq);
+        if (rc) return rc;
+    } else {
+        // V first: metric, selection and V's compaction on stream_v; Q and K follow on
+        // stream_qk as soon as the index list exists.
+        ForkJoin *fj = nullptr;
+        rc = get_events(&fj);
+        if (rc) return rc;
+        CK(cudaEventRecord(fj->fork, sq));
+        CK(cudaStreamWaitEvent(sv, fj->fork, 0));
+        rc = enqueue_metric_select(prev_v, v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, sv);
+        if (rc) return rc;
+        CK(cudaEventRecord(fj->fork, sv));
+        CK(cudaStreamWaitEvent(sq, fj->fork, 0));
+        const uint16_t *in_v[3] = {nullptr, nullptr, v};
+        uint16_t *out_v[3] = {nullptr, nullptr, v_compact};
+        rc = enqueue_pack(in_v, out_v, nullptr, nullptr, 0.f, nullptr, idx, n_active, slots, S, H, D, T, sv);
+        if (rc) return rc;
+        const uint16_t *in_qk[3] = {q, k, nullptr};
+        uint16_t *out_qk[3] = {q_compact, k_compact, nullptr};
+        rc = enqueue_pack(in_qk, out_qk, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T, sq);
+        if (rc) return rc;
+        CK(cudaEventRecord(fj->join, sv));
+        CK(cudaStreamWaitEvent(sq, fj->join, 0));
+    }
+    if (do_unpack) return enqueue_unpack(comp_in, cache, idx, n_active, slots, S, H, D, T, sq);
     return COCODIFF_OK;
 }
 

@@ -16,7 +16,6 @@
 namespace cocodiff {
 namespace {
 
-constexpr int kThreads = 256;
 
 __device__ __forceinline__ void unpack8(const uint4 v, float (&x)[8]) {
     x[0] = __uint_as_float(v.x << 16);
@@ -35,6 +34,13 @@ __device__ __forceinline__ unsigned pack2(float lo, float hi) {
     return *reinterpret_cast<const unsigned *>(&b);
 }
 
+// 1/sqrt(x) for x > 0 (x = mean square + eps): one MUFU, relative error < 2^-22
+__device__ __forceinline__ float rsqrt_approx(float x) {
+    float y;
+    asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 template <int LPR>
 __device__ __forceinline__ float group_sum(float v, unsigned mask) {
 #pragma unroll
@@ -48,15 +54,35 @@ enum JobKind : int { KIND_PLAIN = 0, KIND_NORM = 1, KIND_MIXED = 2 };
 
 // LPR lanes per row (D = 8 * LPR), UN / UP = heads in flight per thread on the
 // norm path / the plain path.
-template <int LPR, int KIND, int UN, int UP>
-__global__ void __launch_bounds__(kThreads, 4) move_rows_kernel(const __grid_constant__ MoveParams p) {
-    constexpr int D = LPR * 8;
-    constexpr int TOK = kThreads / LPR;  // token slots per block
+// THREADS x MINB = threads resident per SM; HINT selects the cache policy of
+// the streaming accesses (0: evict-first loads and stores, 1: read-only path
+// loads + evict-first stores, 2: default).
+template <int HINT>
+__device__ __forceinline__ uint4 ld_row(const uint4 *p) {
+    if (HINT == 0) return __ldcs(p);
+    if (HINT == 1) return __ldg(p);
+    return *p;
+}
+template <int HINT>
+__device__ __forceinline__ void st_row(uint4 *p, const uint4 v) {
+    if (HINT == 2) *p = v; else __stcs(p, v);
+}
 
-    const int tiles = (p.n_slots + TOK - 1) / TOK;
-    const int job_i = blockIdx.x / tiles;
-    const int tile = blockIdx.x - job_i * tiles;
-    const MoveJob job = job_i == 0 ? p.job[0] : (job_i == 1 ? p.job[1] : p.job[2]);
+template <int U>
+struct UnrollTag { static constexpr int value = U; };
+
+// Walks heads [h, h_hi) in groups of U (all loads of a group are issued before
+// its stores), then halves U for what is left, down to single heads.
+template <int U, typename F>
+__device__ __forceinline__ void heads_loop(int &h, const int h_hi, F &&body) {
+    for (; h + U <= h_hi; h += U) body(UnrollTag<U>{});
+    if constexpr (U > 1) heads_loop<U / 2>(h, h_hi, body);
+}
+
+template <int LPR, int KIND, int UN, int UP, int THREADS, int MINB, int HINT>
+__global__ void __launch_bounds__(THREADS, MINB) move_rows_kernel(const __grid_constant__ MoveParams p) {
+    constexpr int D = LPR * 8;
+    constexpr int TOK = THREADS / LPR;  // token slots per tile
 
     int n_valid = p.n_slots;
     long long src_head = p.src_head, dst_head = p.dst_head;
@@ -67,96 +93,142 @@ __global__ void __launch_bounds__(kThreads, 4) move_rows_kernel(const __grid_con
         if (src_head == COMPACT_STRIDE) src_head = (long long)n_valid * D;
         if (dst_head == COMPACT_STRIDE) dst_head = (long long)n_valid * D;
     }
-
-    const int o = tile * TOK + (int)threadIdx.x / LPR;
-    const int lr = (int)threadIdx.x % LPR;
-    if (o >= n_valid) return;  // whole LPR-lane groups leave together
-
-    long long s = o, d = o;
-    if (p.map != MAP_FULL) {
-        const int a = o / p.T;
-        const long long t = (long long)__ldg(p.idx + a) * p.T + (o - a * p.T);
-        if (p.map == MAP_GATHER) s = t; else d = t;
-    }
-
-    const uint4 *sp = reinterpret_cast<const uint4 *>(job.src + s * p.src_tok) + lr;
-    uint4 *dp = reinterpret_cast<uint4 *>(job.dst + d * p.dst_tok) + lr;
     const long long sh = src_head / 8, dh = dst_head / 8;  // head strides in vectors
-    const int H = p.H;
-
-    if (KIND == KIND_PLAIN || (KIND == KIND_MIXED && job.w == nullptr)) {
-        int h = 0;
-        for (; h + UP <= H; h += UP) {
-            uint4 v[UP];
-#pragma unroll
-            for (int u = 0; u < UP; ++u) { v[u] = __ldcs(sp); sp += sh; }
-#pragma unroll
-            for (int u = 0; u < UP; ++u) { __stcs(dp, v[u]); dp += dh; }
-        }
-        for (; h < H; ++h) { __stcs(dp, __ldcs(sp)); sp += sh; dp += dh; }
-        return;
-    }
-
-    float w[8];
-    unpack8(__ldg(reinterpret_cast<const uint4 *>(job.w) + lr), w);
-    float c[4] = {1.f, 1.f, 1.f, 1.f}, sn[4] = {0.f, 0.f, 0.f, 0.f};
-    if (p.cs != nullptr) {
-        // pairs 4*lr .. 4*lr+3 of token s: 8 floats (cos, sin, cos, sin, ...)
-        const float4 *t = reinterpret_cast<const float4 *>(p.cs + s * D) + 2 * lr;
-        const float4 t0 = __ldg(t), t1 = __ldg(t + 1);
-        c[0] = t0.x; sn[0] = t0.y; c[1] = t0.z; sn[1] = t0.w;
-        c[2] = t1.x; sn[2] = t1.y; c[3] = t1.z; sn[3] = t1.w;
-    }
+    const int lr = (int)threadIdx.x % LPR;
     const unsigned lane = threadIdx.x & 31u;
     const unsigned gmask = LPR == 32 ? 0xffffffffu : (((1u << LPR) - 1u) << (lane & ~(unsigned)(LPR - 1)));
-    const float inv_d = 1.0f / (float)D;
-    const float eps = p.eps;
 
-    auto norm_rope_row = [&](const uint4 v) -> uint4 {
-        float x[8];
-        unpack8(v, x);
-        float ss = 0.f;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) ss = fmaf(x[j], x[j], ss);
-        ss = group_sum<LPR>(ss, gmask);
-        const float inv = 1.0f / sqrtf(fmaf(ss, inv_d, eps));
-        unsigned out[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const float a = x[2 * q] * inv * w[2 * q];
-            const float b = x[2 * q + 1] * inv * w[2 * q + 1];
-            out[q] = pack2(a * c[q] - b * sn[q], a * sn[q] + b * c[q]);
+    // The heads of a tile may be split over `head_split` blocks.  Block order:
+    // split-major (all tiles of head range 0 first) or tile-major.
+    const int hsplit = p.head_split > 1 ? p.head_split : 1;
+    const int hs = (p.H + hsplit - 1) / hsplit;
+    const int tiles = (p.n_slots + TOK - 1) / TOK;  // per job; V's tiles come first in the grid
+    const int tiles_all = tiles * p.njobs;
+    const long long total = (long long)tiles_all * hsplit;
+    for (long long b = blockIdx.x; b < total; b += gridDim.x) {
+        int t, y;
+        if (p.tile_major) { t = (int)(b / hsplit); y = (int)(b - (long long)t * hsplit); }
+        else { y = (int)(b / tiles_all); t = (int)(b - (long long)y * tiles_all); }
+        const int h_lo = y * hs;
+        const int h_hi = h_lo + hs < p.H ? h_lo + hs : p.H;
+        const int job_i = t / tiles;
+        const int tile = t - job_i * tiles;
+        const MoveJob job = job_i == 0 ? p.job[0] : (job_i == 1 ? p.job[1] : p.job[2]);
+
+        const int o = tile * TOK + (int)threadIdx.x / LPR;
+        if (o >= n_valid) continue;  // whole LPR-lane groups skip together
+
+        long long s = o, d = o;
+        if (p.map != MAP_FULL) {
+            const int a = o / p.T;
+            const long long tk = (long long)__ldg(p.idx + a) * p.T + (o - a * p.T);
+            if (p.map == MAP_GATHER) s = tk; else d = tk;
         }
-        return make_uint4(out[0], out[1], out[2], out[3]);
-    };
+        const uint4 *sp = reinterpret_cast<const uint4 *>(job.src + s * p.src_tok) + lr + h_lo * sh;
+        uint4 *dp = reinterpret_cast<uint4 *>(job.dst + d * p.dst_tok) + lr + h_lo * dh;
 
-    int h = 0;
-    for (; h + UN <= H; h += UN) {
-        uint4 v[UN];
+        if (KIND == KIND_PLAIN || (KIND == KIND_MIXED && job.w == nullptr)) {
+            int h = h_lo;
+            heads_loop<UP>(h, h_hi, [&](auto u_tag) {
+                constexpr int U = decltype(u_tag)::value;
+                uint4 v[U];
 #pragma unroll
-        for (int u = 0; u < UN; ++u) { v[u] = __ldcs(sp); sp += sh; }
+                for (int u = 0; u < U; ++u) { v[u] = ld_row<HINT>(sp); sp += sh; }
 #pragma unroll
-        for (int u = 0; u < UN; ++u) { __stcs(dp, norm_rope_row(v[u])); dp += dh; }
+                for (int u = 0; u < U; ++u) { st_row<HINT>(dp, v[u]); dp += dh; }
+            });
+            continue;
+        }
+
+        // Per-token constants, reused for all heads: the norm weight folded into the
+        // rotation.  out[2q] = inv*(x[2q]*ka - x[2q+1]*kb), out[2q+1] = inv*(x[2q]*kc + x[2q+1]*kd).
+        float ka[4], kb[4], kc[4], kd[4];
+        {
+            float w[8];
+            unpack8(__ldg(reinterpret_cast<const uint4 *>(job.w) + lr), w);
+            float c[4] = {1.f, 1.f, 1.f, 1.f}, sn[4] = {0.f, 0.f, 0.f, 0.f};
+            if (p.cs != nullptr) {
+                // pairs 4*lr .. 4*lr+3 of token s: 8 floats (cos, sin, cos, sin, ...)
+                const float4 *tb = reinterpret_cast<const float4 *>(p.cs + s * D) + 2 * lr;
+                const float4 t0 = __ldg(tb), t1 = __ldg(tb + 1);
+                c[0] = t0.x; sn[0] = t0.y; c[1] = t0.z; sn[1] = t0.w;
+                c[2] = t1.x; sn[2] = t1.y; c[3] = t1.z; sn[3] = t1.w;
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                ka[q] = w[2 * q] * c[q];
+                kb[q] = w[2 * q + 1] * sn[q];
+                kc[q] = w[2 * q] * sn[q];
+                kd[q] = w[2 * q + 1] * c[q];
+            }
+        }
+        const float inv_d = 1.0f / (float)D;
+        const float eps = p.eps;
+
+        auto norm_rope_row = [&](const uint4 v) -> uint4 {
+            float x[8];
+            unpack8(v, x);
+            float ss = x[0] * x[0];
+#pragma unroll
+            for (int j = 1; j < 8; ++j) ss = fmaf(x[j], x[j], ss);
+            ss = group_sum<LPR>(ss, gmask);
+            const float inv = rsqrt_approx(fmaf(ss, inv_d, eps));
+            unsigned out[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float lo = fmaf(x[2 * q], ka[q], -(x[2 * q + 1] * kb[q])) * inv;
+                const float hi = fmaf(x[2 * q], kc[q], x[2 * q + 1] * kd[q]) * inv;
+                out[q] = pack2(lo, hi);
+            }
+            return make_uint4(out[0], out[1], out[2], out[3]);
+        };
+
+        int h = h_lo;
+        heads_loop<UN>(h, h_hi, [&](auto u_tag) {
+            constexpr int U = decltype(u_tag)::value;
+            uint4 v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) { v[u] = ld_row<HINT>(sp); sp += sh; }
+#pragma unroll
+            for (int u = 0; u < U; ++u) { st_row<HINT>(dp, norm_rope_row(v[u])); dp += dh; }
+        });
     }
-    for (; h < H; ++h) { __stcs(dp, norm_rope_row(__ldcs(sp))); sp += sh; dp += dh; }
 }
 
-template <int LPR>
-cudaError_t launch_lpr(const MoveParams &p, cudaStream_t stream) {
-    constexpr int TOK = kThreads / LPR;
+// Tuned launch shape (see the tuning notes in the design document).
+constexpr int kThreads = 256, kMinBlocks = 4, kUN = 4, kUP = 8, kHint = 0;
+
+// max_blocks > 0 caps the grid (blocks then loop over tiles); head_split > 1
+// spreads the heads of a tile over that many blocks.
+template <int LPR, int KIND, int UN, int UP, int THREADS, int MINB, int HINT>
+cudaError_t launch_variant(MoveParams p, cudaStream_t stream, long long max_blocks = 0, int head_split = 1,
+                           int tile_major = 0) {
+    constexpr int TOK = THREADS / LPR;
     const long long tiles = ((long long)p.n_slots + TOK - 1) / TOK;
-    const long long blocks = tiles * p.njobs;
+    if (head_split < 1) head_split = 1;
+    if (head_split > p.H) head_split = p.H;
+    p.head_split = head_split;
+    p.tile_major = tile_major;
+    long long blocks = tiles * p.njobs * head_split;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    if (max_blocks > 0 && blocks > max_blocks) blocks = max_blocks;
+    move_rows_kernel<LPR, KIND, UN, UP, THREADS, MINB, HINT><<<(unsigned)blocks, THREADS, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+// About eight heads per block measured best on B200 at H = 24 (more blocks per
+// tile: shorter tail, same bytes in flight per thread).
+template <int LPR>
+cudaError_t launch_lpr(const MoveParams &p, cudaStream_t stream) {
     int n_norm = 0;
     for (int i = 0; i < p.njobs; ++i) n_norm += p.job[i].w != nullptr;
+    const int split = (p.H + 7) / 8;
     if (n_norm == 0)
-        move_rows_kernel<LPR, KIND_PLAIN, 4, 8><<<(unsigned)blocks, kThreads, 0, stream>>>(p);
-    else if (n_norm == p.njobs)
-        move_rows_kernel<LPR, KIND_NORM, 4, 8><<<(unsigned)blocks, kThreads, 0, stream>>>(p);
-    else
-        move_rows_kernel<LPR, KIND_MIXED, 4, 8><<<(unsigned)blocks, kThreads, 0, stream>>>(p);
-    return cudaGetLastError();
+        return launch_variant<LPR, KIND_PLAIN, kUN, kUP, kThreads, kMinBlocks, kHint>(p, stream, 0, split);
+    if (n_norm == p.njobs)
+        return launch_variant<LPR, KIND_NORM, kUN, kUP, kThreads, kMinBlocks, kHint>(p, stream, 0, split);
+    return launch_variant<LPR, KIND_MIXED, kUN, kUP, kThreads, kMinBlocks, kHint>(p, stream, 0, split);
 }
 
 }  // namespace

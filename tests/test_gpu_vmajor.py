@@ -224,3 +224,71 @@ def test_temporal_steps_select_compact_unpack(small):
             cache[x].t.copy_(dev(cache_ref[x]).reshape(-1))     # re-align the two sides bit for bit
             cache[x].assert_guards()
         prev_v = cur["v"]
+
+
+@pytest.mark.parametrize("order,two_streams", [(binding.LUMP, False), (binding.V_FIRST, True), (binding.V_FIRST, False)])
+@pytest.mark.parametrize("P,S,H,D,T,r,n_groups", [(4, 768, 4, 64, 16, 0.8, 1), (2, 256, 6, 128, 1, 0.5, 2),
+                                                   (3, 99, 3, 32, 11, 0.0, 1), (2, 384, 2, 256, 64, 1.0, 1)])
+def test_selective_prologue_one_call(order, two_streams, P, S, H, D, T, r, n_groups):
+    """The fused selective step equals the oracle's select -> extract -> scatter,
+    and the batched pack / unpack entry points equal the single-tensor ones."""
+    E, n = S * H * D, S // T
+    rng = np.random.default_rng(S + T)
+    prev, cur_v, _ = _pair(S, H, D, T, seed=S)
+    x = {"q": synth.normal_bf16(8, "q", E).reshape(S, H, D), "k": synth.normal_bf16(8, "k", E).reshape(S, H, D),
+         "v": cur_v}
+    w = {"q": synth.normal_bf16(8, "wq", D, 1.0, 0.1), "k": synth.normal_bf16(8, "wk", D, 1.0, 0.1)}
+    pos = rng.integers(0, 150, (S, 2)).astype(np.int32)
+    cs_ref, cs = oracle.rope_table_2d(pos, D, 10000.0), rope_table(pos, D, 10000.0)
+    old = {t: synth.normal_bf16(9, "old" + t, E).reshape(H, S, D) for t in "qkv"}
+    comp = {t: Guarded(E) for t in "qkv"}
+    cache = {t: Guarded(E, fill=old[t]) for t in "qkv"}
+    sel = Selector(P, S, H, D, T)
+    d = {t: dev(x[t]) for t in "qkv"}
+    sq = torch.cuda.Stream()
+    sv = torch.cuda.Stream() if two_streams else sq
+    torch.cuda.synchronize()
+    binding.selective_prologue(dev(prev), d["q"], d["k"], d["v"], dev(w["q"]), dev(w["k"]), 1e-6, cs, P, S, H, D, T,
+                               r, n_groups, sel.metric, sel.mask, sel.idx, sel.n_active,
+                               comp["q"].t, comp["k"].t, comp["v"].t, cache["q"].t, cache["k"].t, cache["v"].t,
+                               sel.ws, sel.ws_bytes, order=order, stream_qk=sq, stream_v=sv)
+    sq.synchronize()
+    m_ref = oracle.vmajor_metric(prev, cur_v, P, T)
+    mask_ref, idx_ref, na_ref = oracle.vmajor_select(m_ref, n_groups, r)
+    assert np.array_equal(sel.metric.cpu().numpy().view(np.uint64)[:n], m_ref)
+    assert int(sel.n_active.item()) == na_ref
+    assert np.array_equal(sel.mask.cpu().numpy()[:n], mask_ref)
+    assert np.array_equal(sel.idx.cpu().numpy()[:na_ref], idx_ref)
+    tok = (idx_ref[:, None] * T + np.arange(T)[None, :]).reshape(-1).astype(np.int64)
+    inactive = np.ones(S, bool)
+    inactive[tok] = False
+    for t in "qkv":
+        if t == "v":
+            ref, ref_f = x["v"], None
+        else:
+            ref, ref_f = oracle.norm_rope(x[t], w[t], 1e-6, cs_ref, want_f32=True)
+        comp_ref = oracle.pack_active(ref, idx_ref, P, T)
+        got_c = comp[t].host()[:comp_ref.size].reshape(comp_ref.shape)
+        want_cache = oracle.unpack(comp_ref, idx_ref, old[t].copy(), P, T)
+        got_cache = cache[t].host((H, S, D))
+        assert np.array_equal(got_cache[:, inactive], want_cache[:, inactive])
+        if t == "v":
+            assert np.array_equal(got_c, comp_ref) and np.array_equal(got_cache, want_cache)
+        elif na_ref:
+            f = np.ascontiguousarray(ref_f[tok].transpose(1, 0, 2))
+            assert_norm_rope_close(got_c, comp_ref, f, t + " compact")
+            assert np.array_equal(got_cache[:, tok], got_c), "scatter moves the compact rows bit-exactly"
+        assert np.all(comp[t].host()[comp_ref.size:] == 0x5A5A)
+        comp[t].assert_guards()
+        cache[t].assert_guards()
+    # batched entry points against the fused call's own outputs
+    comp2 = {t: Guarded(E) for t in "qkv"}
+    cache2 = {t: Guarded(E, fill=old[t]) for t in "qkv"}
+    binding.pack_active_qkv(d["q"], d["k"], d["v"], dev(w["q"]), dev(w["k"]), 1e-6, cs, sel.idx, sel.n_active,
+                            comp2["q"].t, comp2["k"].t, comp2["v"].t, P, S, H, D, T)
+    binding.unpack_qkv(comp2["q"].t, comp2["k"].t, comp2["v"].t, sel.idx, sel.n_active,
+                       cache2["q"].t, cache2["k"].t, cache2["v"].t, P, S, H, D, T)
+    torch.cuda.synchronize()
+    for t in "qkv":
+        assert np.array_equal(comp2[t].host(), comp[t].host())
+        assert np.array_equal(cache2[t].host(), cache[t].host())
