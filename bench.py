@@ -333,7 +333,7 @@ def read_traffic_note():
         return None
 
 
-def other_configs(torch, binding, args):
+def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "temporal")):
     """µs/layer and GB/s of the other synthetic workloads, L2 flushed between
     iterations (they fit in the 126 MB L2), plus the selective step of the
     temporal workload."""
@@ -346,7 +346,7 @@ def other_configs(torch, binding, args):
             scratch.zero_()
 
     iters = max(10, min(args.steps, 50))
-    for name in ("tiny", "sd3", "qwen768", "temporal"):
+    for name in names:
         cfg = synth.config(name)
         P, S, H, D = cfg["P"], cfg["S"], cfg["H"], cfg["D"]
         E = S * H * D
@@ -412,9 +412,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--only-main", action="store_true",
                     help="run only the headline loop (short launch list for profiling)")
+    ap.add_argument("--only-temporal", action="store_true",
+                    help="run only the temporal workload (full step and selective step), for profiling")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.only_temporal:
+        import torch
+        from paper_2604_14561_b200 import binding
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        print(json.dumps({"per_config": other_configs(torch, binding, args, names=("temporal",))}, ensure_ascii=False))
     else:
         run_ours(args)
 
