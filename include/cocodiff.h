@@ -194,6 +194,38 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
                                 void *workspace, size_t workspace_bytes, cocodiff_order order,
                                 void *stream_qk, void *stream_v);
 
+/* cocodiff_vmajor_select_compact for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a deployment convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a plug-in inside
+ * a serving process whose memory pool is owned by someone else, a hook that runs
+ * while the application is in a no-allocation phase, a real-time loop that must
+ * not touch the allocator.  Such callers already own their inputs and outputs
+ * but have nowhere to get the small scratch area the fused metric + selection
+ * kernel needs (per-unit accumulators and a block ticket).  Here that scratch is
+ * a fixed array inside the library image on the device: COCODIFF_STATIC_MAX_UNITS
+ * 64-bit accumulators plus 256 bytes (about 256 KB), present on every GPU that
+ * loads the library until the process exits.
+ *
+ * Arguments and results are exactly those of cocodiff_vmajor_select_compact
+ * without `workspace` / `workspace_bytes`.  Differences to know about:
+ *   - S / T may not exceed COCODIFF_STATIC_MAX_UNITS; more units are refused
+ *     with COCODIFF_WORKSPACE_TOO_SMALL and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current) and remembers it.  Make that first call outside any
+ *     stream capture.
+ *   - Every call on a device shares the one array, which still holds whatever
+ *     the previous call left; each call clears the part it is going to use, on
+ *     its stream, before its kernel runs.  Two calls whose work overlaps on the
+ *     GPU (different streams, no ordering between them) race on the array and
+ *     give wrong selections: order them, or use the workspace-taking call.
+ *   - No cudaMalloc, cudaFree or other allocating routine is called. */
+#define COCODIFF_STATIC_MAX_UNITS 32768
+int cocodiff_vmajor_select_compact_static(const uint16_t *prev_v, const uint16_t *cur_v,
+                                          int P, int S, int H, int D, int T, double r, int n_groups,
+                                          uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
+                                          uint16_t *v_compact, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

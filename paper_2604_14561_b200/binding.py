@@ -41,6 +41,7 @@ SIGNATURES = {
     "cocodiff_unpack": (_I, [_P, _P, _P, _P] + [_I] * 5 + [_P]),
     "cocodiff_pack_active_qkv": (_I, [_P] * 5 + [_F] + [_P] * 6 + [_I] * 5 + [_P]),
     "cocodiff_unpack_qkv": (_I, [_P] * 8 + [_I] * 5 + [_P]),
+    "cocodiff_vmajor_select_compact_static": (_I, [_P, _P] + [_I] * 5 + [_D, _I] + [_P] * 5 + [_P]),
     "cocodiff_selective_prologue": (_I, [_P] * 6 + [_F, _P] + [_I] * 5 + [_D, _I] + [_P] * 11 + [_Z, _I, _P, _P]),
 }
 
@@ -186,3 +187,17 @@ def selective_prologue(prev_v, q, k, v, wq, wk, eps, cs, P, S, H, D, T, r, n_gro
                  _ptr(n_active), _ptr(q_compact), _ptr(k_compact), _ptr(v_compact), _ptr(q_cache),
                  _ptr(k_cache), _ptr(v_cache), _ptr(workspace), workspace_bytes, order,
                  _stream(stream_qk), _stream(stream_v), check=check)
+
+
+STATIC_MAX_UNITS = 32768
+
+
+def vmajor_select_compact_static(prev_v, cur_v, P, S, H, D, T, r, n_groups, metric, mask, idx, n_active,
+                                 v_compact, stream=None, check=True):
+    """`vmajor_select_compact` without a workspace argument, for callers that cannot
+    allocate device memory: the scratch is a fixed array inside the library (at most
+    STATIC_MAX_UNITS selection units).  Calls on one device share that array, so calls
+    that may overlap on the GPU must be ordered by the caller."""
+    return _call("cocodiff_vmajor_select_compact_static", _ptr(prev_v), _ptr(cur_v), P, S, H, D, T, r,
+                 n_groups, _ptr(metric), _ptr(mask), _ptr(idx), _ptr(n_active), _ptr(v_compact),
+                 _stream(stream), check=check)

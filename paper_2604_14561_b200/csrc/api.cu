@@ -3,6 +3,7 @@
 // lives here and no device memory is allocated here.
 #include <cmath>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/cocodiff.h"
 #include "common.cuh"
@@ -587,6 +588,60 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
         CK(cudaStreamWaitEvent(sq, fj->join, 0));
     }
     if (do_unpack) return enqueue_unpack(comp_in, cache, idx, n_active, slots, S, H, D, T, sq);
+    return COCODIFF_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Scratch that lives in the library image, for callers that cannot allocate.
+// One array per GPU that loads the library, held until the process exits.
+#define COCODIFF_STATIC_MAX_UNITS_IMPL 32768
+constexpr size_t kStaticScratchBytes = (size_t)COCODIFF_STATIC_MAX_UNITS_IMPL * 8 + 256;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not a device
+// address; the address is looked up once per device, with that device current.
+static std::mutex g_static_mutex;
+static void *g_static_addr[kMaxDevices];
+
+static int static_scratch_address(void **out) {
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return COCODIFF_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_addr[dev]) {
+        void *ptr = nullptr;
+        CK(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        if (!ptr || (reinterpret_cast<uintptr_t>(ptr) & 255u)) return COCODIFF_MISALIGNED;
+        g_static_addr[dev] = ptr;
+    }
+    *out = g_static_addr[dev];
+    return COCODIFF_OK;
+}
+
+int cocodiff_vmajor_select_compact_static(const uint16_t *prev_v, const uint16_t *cur_v, int P, int S, int H,
+                                          int D, int T, double r, int n_groups, uint64_t *metric,
+                                          uint8_t *mask, int32_t *idx, int32_t *n_active,
+                                          uint16_t *v_compact, void *stream) {
+    // the unit count is checked against the fixed capacity before anything else is looked at
+    if (T >= 1 && S >= 0 && S / T > COCODIFF_STATIC_MAX_UNITS_IMPL) return COCODIFF_WORKSPACE_TOO_SMALL;
+    void *scratch = nullptr;
+    int rc = static_scratch_address(&scratch);
+    if (rc) return rc;
+    rc = check_select(prev_v, cur_v, P, S, H, D, T, r, n_groups, metric, mask, idx, n_active, scratch,
+                      kStaticScratchBytes);
+    if (rc) return rc;
+    const uint16_t *in[3] = {nullptr, nullptr, cur_v};
+    uint16_t *out[3] = {nullptr, nullptr, v_compact};
+    if (v_compact) {
+        rc = check_tiles(in, out, S, H, D, idx, n_active);
+        if (rc) return rc;
+        if (overlap(prev_v, (size_t)S * H * D * 2, v_compact, (size_t)S * H * D * 2)) return COCODIFF_ALIASING;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    // enqueue_metric_select clears the accumulators and the ticket it is about to use
+    rc = enqueue_metric_select(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, scratch, st);
+    if (rc) return rc;
+    if (v_compact) return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, S, S, H, D, T, st);
     return COCODIFF_OK;
 }
 
