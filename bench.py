@@ -261,13 +261,18 @@ def run_ours(args):
             orders[name] = {"us_median": 1e3 * statistics.median(ms), "us_min": 1e3 * min(ms),
                             "gbs_median": step_bytes / (statistics.median(ms) * 1e-3) / 1e9,
                             "launches_per_step": 2 if order == binding.V_FIRST else 1}
-        # dominant kernel: move_rows_kernel, timed where one launch is the whole step (lump order)
-        lump_ms = statistics.mean(time_steps(torch, lambda: step(binding.LUMP), sq, args.steps, 3))
-        achieved = step_bytes / (lump_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": "move_rows_kernel<LPR=16, mixed> (Q,K norm+RoPE+exchange and V exchange in one launch)",
+        # dominant kernel of the headline loop: the norm + RoPE + exchange launch over Q and K
+        # (two thirds of the bytes), timed alone on its stream
+        def qk_only():
+            binding.prologue(q, k, None, qh, kh, None, wq, wk, cfg["eps"], cs, P, S, H, D, order=binding.V_FIRST,
+                             stream_qk=sq, stream_v=sv)
+        qk_ms = statistics.mean(time_steps(torch, qk_only, sq, args.steps, 3))
+        qk_bytes = step_bytes * 2 // 3
+        achieved = qk_bytes / (qk_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "move_rows_kernel<LPR=16, KIND_NORM> (Q and K: RMSNorm + RoPE + exchange, one launch)",
                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                     "frac": achieved / peak, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                    "us_per_launch": 1e3 * lump_ms, "algorithmic_bytes_per_launch": step_bytes,
+                    "us_per_launch": 1e3 * qk_ms, "algorithmic_bytes_per_launch": qk_bytes,
                     "traffic": read_traffic_note()}
 
         # ---- end to end: host buffers in, host buffers out ------------------
@@ -328,7 +333,7 @@ def read_traffic_note():
     path = os.path.join(ROOT, "profiles", "traffic.json")
     try:
         with open(path) as f:
-            return json.load(f).get("move_rows_mixed_qwen2304_bytes_per_launch")
+            return json.load(f).get("move_rows_norm_qwen2304_dram_bytes_per_launch")
     except Exception:
         return None
 

@@ -95,7 +95,8 @@ int cocodiff_ulysses_a2a_inverse(const uint16_t *q_head, const uint16_t *k_head,
 /* The fused prologue of one layer, full exchange (Sections II-B, II-A, III-C):
  * every (token, head) row of Q and K is read once, normalised, rotated and
  * written straight into its HEAD slot; V is moved untouched, first.  Stream
- * semantics as for cocodiff_ulysses_a2a.  All six tensors are required. */
+ * semantics as for cocodiff_ulysses_a2a.  A (x, x_head) pair may be NULL/NULL to
+ * leave that tensor out (a layer normally passes all three). */
 int cocodiff_prologue(const uint16_t *q, const uint16_t *k, const uint16_t *v,
                       uint16_t *q_head, uint16_t *k_head, uint16_t *v_head,
                       const uint16_t *wq, const uint16_t *wk, float eps, const float *cs,

@@ -350,8 +350,7 @@ int cocodiff_prologue(const uint16_t *q, const uint16_t *k, const uint16_t *v, u
     int rc = check_shape(P, S, H, D);
     if (rc) return rc;
     if (order != COCODIFF_LUMP && order != COCODIFF_V_FIRST) return COCODIFF_INVALID_ARG;
-    if (!q || !k || !v || !q_head || !k_head || !v_head || !wq || !wk || !cs || !(eps >= 0.f))
-        return COCODIFF_INVALID_ARG;
+    if ((q && !wq) || (k && !wk) || ((q || k) && !cs) || !(eps >= 0.f)) return COCODIFF_INVALID_ARG;
     if (!aligned16(wq) || !aligned16(wk) || !aligned16(cs)) return COCODIFF_MISALIGNED;
     const uint16_t *in[3] = {q, k, v};
     uint16_t *out[3] = {q_head, k_head, v_head};

@@ -65,6 +65,8 @@ def test_pointer_validation():
     assert binding.ulysses_a2a(q, k, v, qh, qh, vh, 2, 8, 4, 64, check=False) == -6         # out/out overlap
     w, cs = _addr(40), _addr(41)
     assert binding.prologue(q, k, v, qh, kh, vh, None, w, 1e-6, cs, 2, 8, 4, 64, check=False) == -1
+    assert binding.prologue(q, k, v, qh, kh, vh, w, w, 1e-6, None, 2, 8, 4, 64, check=False) == -1
+    assert binding.prologue(q, k, None, qh, kh, vh, w, w, 1e-6, cs, 2, 8, 4, 64, check=False) == -1
     assert binding.prologue(q, k, v, qh, kh, vh, w, w, -1.0, cs, 2, 8, 4, 64, check=False) == -1
     assert binding.prologue(q, k, v, qh, kh, vh, w, w, 1e-6, cs + 4, 2, 8, 4, 64, check=False) == -3
     # norm + rope in place is allowed to alias exactly, not partially
