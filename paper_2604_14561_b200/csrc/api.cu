@@ -179,7 +179,7 @@ int enqueue_metric_select(const uint16_t *prev_v, const uint16_t *cur_v, int S, 
     mp.ticket = reinterpret_cast<unsigned int *>(reinterpret_cast<char *>(workspace) + (need - 256));
     mp.metric = reinterpret_cast<unsigned long long *>(metric);
     mp.unit_vecs = (long long)T * H * D / 8;
-    mp.chunk_vecs = 512;
+    mp.chunk_vecs = 128;  // 2 KB of each tensor per warp visit: one group of loads in flight
     mp.chunks_per_unit = (int)((mp.unit_vecs + mp.chunk_vecs - 1) / mp.chunk_vecs);
     mp.n_units = n;
     mp.sel.metric = mp.metric;

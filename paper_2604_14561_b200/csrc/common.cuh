@@ -35,8 +35,8 @@ struct MoveParams {
     const int32_t *n_active;
     int T;
     int map;
-    int head_split;         // blocks per tile along the heads (>= 1)
-    int tile_major;         // block order when head_split > 1
+    int head_split;         // blocks per tile along the heads (>= 1); set by the launcher
+    int order;              // block order; set by the launcher
 };
 
 struct SelectParams {

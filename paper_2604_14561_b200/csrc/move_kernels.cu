@@ -41,10 +41,11 @@ __device__ __forceinline__ float rsqrt_approx(float x) {
     return y;
 }
 
+// Sum over the LPR lanes that hold one row; the whole warp takes part.
 template <int LPR>
-__device__ __forceinline__ float group_sum(float v, unsigned mask) {
+__device__ __forceinline__ float group_sum(float v) {
 #pragma unroll
-    for (int off = LPR / 2; off >= 1; off >>= 1) v += __shfl_xor_sync(mask, v, off);
+    for (int off = LPR / 2; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
     return v;
 }
 
@@ -89,146 +90,152 @@ __global__ void __launch_bounds__(THREADS, MINB) move_rows_kernel(const __grid_c
     if (p.map != MAP_FULL) {
         const long long nv = (long long)__ldg(p.n_active) * p.T;
         n_valid = nv < (long long)p.n_slots ? (int)nv : p.n_slots;
-        if (n_valid < 0) n_valid = 0;
         if (src_head == COMPACT_STRIDE) src_head = (long long)n_valid * D;
         if (dst_head == COMPACT_STRIDE) dst_head = (long long)n_valid * D;
     }
+    // Block id -> (job, head range, token tile).  ORDER 0: job-major (all of V,
+    // then Q, then K); 1: head-range-major (V, Q, K tiles of range 0, then range 1 ...);
+    // 2: tile-major (the jobs and ranges of one tile are neighbours).
+    const unsigned tiles = (unsigned)(p.n_slots + TOK - 1) / TOK;
+    const unsigned hsplit = (unsigned)p.head_split, njobs = (unsigned)p.njobs;
+    unsigned tile, y, job_i;
+    {
+        const unsigned b = blockIdx.x;
+        if (p.order == 0) { job_i = b / (tiles * hsplit); const unsigned r = b - job_i * tiles * hsplit; y = r / tiles; tile = r - y * tiles; }
+        else if (p.order == 1) { y = b / (tiles * njobs); const unsigned r = b - y * tiles * njobs; job_i = r / tiles; tile = r - job_i * tiles; }
+        else { tile = b / (njobs * hsplit); const unsigned r = b - tile * njobs * hsplit; job_i = r / hsplit; y = r - job_i * hsplit; }
+    }
+    const int tile0 = (int)tile * TOK;
+    if (tile0 >= n_valid) return;  // block-uniform: nothing in this tile
     const long long sh = src_head / 8, dh = dst_head / 8;  // head strides in vectors
     const int lr = (int)threadIdx.x % LPR;
-    const unsigned lane = threadIdx.x & 31u;
-    const unsigned gmask = LPR == 32 ? 0xffffffffu : (((1u << LPR) - 1u) << (lane & ~(unsigned)(LPR - 1)));
 
-    // The heads of a tile may be split over `head_split` blocks.  Block order:
-    // split-major (all tiles of head range 0 first) or tile-major.
-    const int hsplit = p.head_split > 1 ? p.head_split : 1;
-    const int hs = (p.H + hsplit - 1) / hsplit;
-    const int tiles = (p.n_slots + TOK - 1) / TOK;  // per job; V's tiles come first in the grid
-    const int tiles_all = tiles * p.njobs;
-    const long long total = (long long)tiles_all * hsplit;
-    for (long long b = blockIdx.x; b < total; b += gridDim.x) {
-        int t, y;
-        if (p.tile_major) { t = (int)(b / hsplit); y = (int)(b - (long long)t * hsplit); }
-        else { y = (int)(b / tiles_all); t = (int)(b - (long long)y * tiles_all); }
-        const int h_lo = y * hs;
-        const int h_hi = h_lo + hs < p.H ? h_lo + hs : p.H;
-        const int job_i = t / tiles;
-        const int tile = t - job_i * tiles;
-        const MoveJob job = job_i == 0 ? p.job[0] : (job_i == 1 ? p.job[1] : p.job[2]);
+    // heads [h_lo, h_hi) of this block
+    const int hs = (p.H + (int)hsplit - 1) / (int)hsplit;
+    const int h_lo = (int)y * hs;
+    const int h_hi = h_lo + hs < p.H ? h_lo + hs : p.H;
+    const MoveJob job = job_i == 0 ? p.job[0] : (job_i == 1 ? p.job[1] : p.job[2]);
 
-        const int o = tile * TOK + (int)threadIdx.x / LPR;
-        if (o >= n_valid) continue;  // whole LPR-lane groups skip together
+    // A slot past the end keeps its lanes in step with the warp (the row
+    // reduction uses full-warp shuffles): it re-reads the tile's first slot
+    // and stores nothing.
+    const int o_raw = tile0 + (int)threadIdx.x / LPR;
+    const bool valid = o_raw < n_valid;
+    const int o = valid ? o_raw : tile0;
 
-        long long s = o, d = o;
-        if (p.map != MAP_FULL) {
-            const int a = o / p.T;
-            const long long tk = (long long)__ldg(p.idx + a) * p.T + (o - a * p.T);
-            if (p.map == MAP_GATHER) s = tk; else d = tk;
-        }
-        const uint4 *sp = reinterpret_cast<const uint4 *>(job.src + s * p.src_tok) + lr + h_lo * sh;
-        uint4 *dp = reinterpret_cast<uint4 *>(job.dst + d * p.dst_tok) + lr + h_lo * dh;
+    long long s = o, d = o;
+    if (p.map != MAP_FULL) {
+        const int a = o / p.T;
+        const long long tk = (long long)__ldg(p.idx + a) * p.T + (o - a * p.T);
+        if (p.map == MAP_GATHER) s = tk; else d = tk;
+    }
+    const uint4 *sp = reinterpret_cast<const uint4 *>(job.src + s * p.src_tok) + lr + h_lo * sh;
+    uint4 *dp = reinterpret_cast<uint4 *>(job.dst + d * p.dst_tok) + lr + h_lo * dh;
 
-        if (KIND == KIND_PLAIN || (KIND == KIND_MIXED && job.w == nullptr)) {
-            int h = h_lo;
-            heads_loop<UP>(h, h_hi, [&](auto u_tag) {
-                constexpr int U = decltype(u_tag)::value;
-                uint4 v[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) { v[u] = ld_row<HINT>(sp); sp += sh; }
-#pragma unroll
-                for (int u = 0; u < U; ++u) { st_row<HINT>(dp, v[u]); dp += dh; }
-            });
-            continue;
-        }
-
-        // Per-token constants, reused for all heads: the norm weight folded into the
-        // rotation.  out[2q] = inv*(x[2q]*ka - x[2q+1]*kb), out[2q+1] = inv*(x[2q]*kc + x[2q+1]*kd).
-        float ka[4], kb[4], kc[4], kd[4];
-        {
-            float w[8];
-            unpack8(__ldg(reinterpret_cast<const uint4 *>(job.w) + lr), w);
-            float c[4] = {1.f, 1.f, 1.f, 1.f}, sn[4] = {0.f, 0.f, 0.f, 0.f};
-            if (p.cs != nullptr) {
-                // pairs 4*lr .. 4*lr+3 of token s: 8 floats (cos, sin, cos, sin, ...)
-                const float4 *tb = reinterpret_cast<const float4 *>(p.cs + s * D) + 2 * lr;
-                const float4 t0 = __ldg(tb), t1 = __ldg(tb + 1);
-                c[0] = t0.x; sn[0] = t0.y; c[1] = t0.z; sn[1] = t0.w;
-                c[2] = t1.x; sn[2] = t1.y; c[3] = t1.z; sn[3] = t1.w;
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                ka[q] = w[2 * q] * c[q];
-                kb[q] = w[2 * q + 1] * sn[q];
-                kc[q] = w[2 * q] * sn[q];
-                kd[q] = w[2 * q + 1] * c[q];
-            }
-        }
-        const float inv_d = 1.0f / (float)D;
-        const float eps = p.eps;
-
-        auto norm_rope_row = [&](const uint4 v) -> uint4 {
-            float x[8];
-            unpack8(v, x);
-            float ss = x[0] * x[0];
-#pragma unroll
-            for (int j = 1; j < 8; ++j) ss = fmaf(x[j], x[j], ss);
-            ss = group_sum<LPR>(ss, gmask);
-            const float inv = rsqrt_approx(fmaf(ss, inv_d, eps));
-            unsigned out[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float lo = fmaf(x[2 * q], ka[q], -(x[2 * q + 1] * kb[q])) * inv;
-                const float hi = fmaf(x[2 * q], kc[q], x[2 * q + 1] * kd[q]) * inv;
-                out[q] = pack2(lo, hi);
-            }
-            return make_uint4(out[0], out[1], out[2], out[3]);
-        };
-
+    if (KIND == KIND_PLAIN || (KIND == KIND_MIXED && job.w == nullptr)) {
+        if (!valid) return;
         int h = h_lo;
-        heads_loop<UN>(h, h_hi, [&](auto u_tag) {
+        heads_loop<UP>(h, h_hi, [&](auto u_tag) {
             constexpr int U = decltype(u_tag)::value;
             uint4 v[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) { v[u] = ld_row<HINT>(sp); sp += sh; }
 #pragma unroll
-            for (int u = 0; u < U; ++u) { st_row<HINT>(dp, norm_rope_row(v[u])); dp += dh; }
+            for (int u = 0; u < U; ++u) { st_row<HINT>(dp, v[u]); dp += dh; }
         });
+        return;
     }
+
+    // Per-token constants, reused for all heads: the norm weight folded into the
+    // rotation.  out[2q] = inv*(x[2q]*ka - x[2q+1]*kb), out[2q+1] = inv*(x[2q]*kc + x[2q+1]*kd).
+    float ka[4], kb[4], kc[4], kd[4];
+    {
+        float w[8];
+        unpack8(__ldg(reinterpret_cast<const uint4 *>(job.w) + lr), w);
+        float c[4] = {1.f, 1.f, 1.f, 1.f}, sn[4] = {0.f, 0.f, 0.f, 0.f};
+        if (p.cs != nullptr) {
+            // pairs 4*lr .. 4*lr+3 of token s: 8 floats (cos, sin, cos, sin, ...)
+            const float4 *tb = reinterpret_cast<const float4 *>(p.cs + s * D) + 2 * lr;
+            const float4 t0 = __ldg(tb), t1 = __ldg(tb + 1);
+            c[0] = t0.x; sn[0] = t0.y; c[1] = t0.z; sn[1] = t0.w;
+            c[2] = t1.x; sn[2] = t1.y; c[3] = t1.z; sn[3] = t1.w;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            ka[q] = w[2 * q] * c[q];
+            kb[q] = -(w[2 * q + 1] * sn[q]);
+            kc[q] = w[2 * q] * sn[q];
+            kd[q] = w[2 * q + 1] * c[q];
+        }
+    }
+    const float inv_d = 1.0f / (float)D;
+    const float eps = p.eps;
+
+    auto norm_rope_row = [&](const uint4 v) -> uint4 {
+        float x[8];
+        unpack8(v, x);
+        float ss = x[0] * x[0];
+#pragma unroll
+        for (int j = 1; j < 8; ++j) ss = fmaf(x[j], x[j], ss);
+        ss = group_sum<LPR>(ss);
+        const float inv = rsqrt_approx(fmaf(ss, inv_d, eps));
+        unsigned out[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float lo = fmaf(x[2 * q], ka[q], x[2 * q + 1] * kb[q]) * inv;
+            const float hi = fmaf(x[2 * q], kc[q], x[2 * q + 1] * kd[q]) * inv;
+            out[q] = pack2(lo, hi);
+        }
+        return make_uint4(out[0], out[1], out[2], out[3]);
+    };
+
+    int h = h_lo;
+    heads_loop<UN>(h, h_hi, [&](auto u_tag) {
+        constexpr int U = decltype(u_tag)::value;
+        uint4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) { v[u] = ld_row<HINT>(sp); sp += sh; }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint4 y = norm_rope_row(v[u]);
+            if (valid) st_row<HINT>(dp, y);
+            dp += dh;
+        }
+    });
 }
 
-// Tuned launch shape (see the tuning notes in the design document).
-constexpr int kThreads = 256, kMinBlocks = 4, kUN = 4, kUP = 8, kHint = 0;
+// Launch shapes measured on B200 at H = 24, D = 128 (21k tokens): 256 threads,
+// 4 blocks per SM (<= 64 registers), evict-first accesses; heads per block and
+// loads in flight per thread depend on what the launch contains.
+constexpr int kThreads = 256, kMinBlocks = 4, kHint = 0;
 
-// max_blocks > 0 caps the grid (blocks then loop over tiles); head_split > 1
-// spreads the heads of a tile over that many blocks.
 template <int LPR, int KIND, int UN, int UP, int THREADS, int MINB, int HINT>
-cudaError_t launch_variant(MoveParams p, cudaStream_t stream, long long max_blocks = 0, int head_split = 1,
-                           int tile_major = 0) {
+cudaError_t launch_variant(MoveParams p, cudaStream_t stream, int head_split = 1, int order = 1) {
     constexpr int TOK = THREADS / LPR;
     const long long tiles = ((long long)p.n_slots + TOK - 1) / TOK;
     if (head_split < 1) head_split = 1;
     if (head_split > p.H) head_split = p.H;
     p.head_split = head_split;
-    p.tile_major = tile_major;
-    long long blocks = tiles * p.njobs * head_split;
+    p.order = order;
+    const long long blocks = tiles * head_split * p.njobs;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    if (max_blocks > 0 && blocks > max_blocks) blocks = max_blocks;
     move_rows_kernel<LPR, KIND, UN, UP, THREADS, MINB, HINT><<<(unsigned)blocks, THREADS, 0, stream>>>(p);
     return cudaGetLastError();
 }
 
-// About eight heads per block measured best on B200 at H = 24 (more blocks per
-// tile: shorter tail, same bytes in flight per thread).
+// Several blocks per token tile shorten the tail of the grid and let V's plain
+// blocks run beside Q/K's arithmetic-heavier ones (head-range-major block order).
 template <int LPR>
 cudaError_t launch_lpr(const MoveParams &p, cudaStream_t stream) {
     int n_norm = 0;
     for (int i = 0; i < p.njobs; ++i) n_norm += p.job[i].w != nullptr;
-    const int split = (p.H + 7) / 8;
-    if (n_norm == 0)
-        return launch_variant<LPR, KIND_PLAIN, kUN, kUP, kThreads, kMinBlocks, kHint>(p, stream, 0, split);
-    if (n_norm == p.njobs)
-        return launch_variant<LPR, KIND_NORM, kUN, kUP, kThreads, kMinBlocks, kHint>(p, stream, 0, split);
-    return launch_variant<LPR, KIND_MIXED, kUN, kUP, kThreads, kMinBlocks, kHint>(p, stream, 0, split);
+    if (n_norm == 0)  // 4 heads per block, 4-8 rows in flight per thread
+        return launch_variant<LPR, KIND_PLAIN, 4, 8, kThreads, kMinBlocks, kHint>(p, stream, (p.H + 3) / 4, 1);
+    if (n_norm == p.njobs)  // 8 heads per block, 4 rows in flight
+        return launch_variant<LPR, KIND_NORM, 4, 8, kThreads, kMinBlocks, kHint>(p, stream, (p.H + 7) / 8, 1);
+    // V with Q and/or K in one launch: 12 heads per block, 4 rows in flight on both paths
+    return launch_variant<LPR, KIND_MIXED, 4, 4, kThreads, kMinBlocks, kHint>(p, stream, (p.H + 11) / 12, 1);
 }
 
 }  // namespace

@@ -160,17 +160,18 @@ __device__ __forceinline__ unsigned long long l1_of_vec(const uint4 a, const uin
     return s;
 }
 
-__global__ void __launch_bounds__(kMetricThreads)
+__global__ void __launch_bounds__(kMetricThreads, 4)
 vmajor_metric_kernel(const __grid_constant__ MetricParams p, const int fuse_select) {
     __shared__ SelectSmem sm;
     __shared__ int is_last;
     constexpr int U = kMetricUnroll;
     const int lane = threadIdx.x & 31;
-    const long long warps = (long long)gridDim.x * (kMetricThreads / 32);
-    const long long total = (long long)p.n_units * p.chunks_per_unit;
-    for (long long c = (long long)blockIdx.x * (kMetricThreads / 32) + (threadIdx.x >> 5); c < total; c += warps) {
-        const int u = (int)(c / p.chunks_per_unit);
-        const int k = (int)(c - (long long)u * p.chunks_per_unit);
+    // chunk ids fit 32 bits (checked by the launcher): no 64-bit divisions here
+    const unsigned warps = gridDim.x * (kMetricThreads / 32);
+    const unsigned total = (unsigned)p.n_units * (unsigned)p.chunks_per_unit;
+    for (unsigned c = blockIdx.x * (kMetricThreads / 32) + (threadIdx.x >> 5); c < total; c += warps) {
+        const unsigned u = c / (unsigned)p.chunks_per_unit;
+        const unsigned k = c - u * (unsigned)p.chunks_per_unit;
         const long long v0 = (long long)k * p.chunk_vecs;
         const long long v1 = v0 + p.chunk_vecs < p.unit_vecs ? v0 + p.chunk_vecs : p.unit_vecs;
         const uint4 *pc = p.cur + (long long)u * p.unit_vecs;
@@ -221,9 +222,13 @@ cudaError_t launch_select(const SelectParams &p, cudaStream_t stream) {
 
 cudaError_t launch_metric_select(const MetricParams &p, cudaStream_t stream) {
     if (p.n_units == 0) return launch_select(p.sel, stream);
+    // One resident wave (4 blocks of 256 threads per SM); its warps walk the chunks.
     const long long total = (long long)p.n_units * p.chunks_per_unit;
+    if (total > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     long long blocks = (total + (kMetricThreads / 32) - 1) / (kMetricThreads / 32);
-    const long long cap = 148LL * 8;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long cap = (long long)sms * 4;
     if (blocks > cap) blocks = cap;
     const int fuse = (p.sel.g <= kCountMax && p.sel.n_groups <= 64) ? 1 : 0;
     vmajor_metric_kernel<<<(unsigned)blocks, kMetricThreads, 0, stream>>>(p, fuse);
