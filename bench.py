@@ -169,6 +169,22 @@ def time_steps(torch, fn, stream, steps, warmup, flush=None):
     return [a.elapsed_time(b) for a, b in ev]
 
 
+def time_loop(torch, fn, stream, steps, warmup=3):
+    """`steps` calls back to back between two CUDA events on `stream`; ms per call."""
+    for _ in range(warmup):
+        fn()
+    stream.synchronize()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(steps):
+        fn()
+    b.record(stream)
+    stream.synchronize()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / steps
+
+
 def max_over_ranks(ms, world, device):
     """The slowest rank's time: every multi-GPU number is the max over ranks."""
     if world <= 1:
@@ -266,7 +282,7 @@ def run_ours(args):
         def qk_only():
             binding.prologue(q, k, None, qh, kh, None, wq, wk, cfg["eps"], cs, P, S, H, D, order=binding.V_FIRST,
                              stream_qk=sq, stream_v=sv)
-        qk_ms = statistics.mean(time_steps(torch, qk_only, sq, args.steps, 3))
+        qk_ms = time_loop(torch, qk_only, sq, args.steps)
         qk_bytes = step_bytes * 2 // 3
         achieved = qk_bytes / (qk_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "move_rows_kernel<LPR=16, KIND_NORM> (Q and K: RMSNorm + RoPE + exchange, one launch)",
