@@ -345,12 +345,14 @@ def run_ours(args):
 
 
 def read_traffic_note():
-    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if present."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
+    """DRAM bytes per launch of the dominant kernel, from the committed ncu summary."""
+    import re
+    path = os.path.join(ROOT, "profiles", "move_rows_kernel_qwen2304.md")
     try:
         with open(path) as f:
-            return json.load(f).get("move_rows_norm_qwen2304_dram_bytes_per_launch")
-    except Exception:
+            m = re.search(r"traffic_bytes_per_launch\(move_rows_norm_qwen2304\)\s*=\s*(\d+)", f.read())
+        return int(m.group(1)) if m else None
+    except OSError:
         return None
 
 
