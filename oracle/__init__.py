@@ -110,6 +110,23 @@ def ulysses_a2a_inverse(head, P):
     return seq
 
 
+def tapa_phase1(seq, P):
+    """seq [S][H][D] -> p1 [2][S][H][D] (p1[t] = the copies held by the tiles of ring t)."""
+    seq = _u16(seq)
+    S, H, D = seq.shape
+    p1 = np.empty((2, S, H, D), dtype=np.uint16)
+    _check(lib().oracle_tapa_phase1(_p(seq), _p(p1), P, S, H, D), "tapa_phase1")
+    return p1
+
+
+def tapa_phase2(p1, P):
+    p1 = _u16(p1)
+    _, S, H, D = p1.shape
+    head = np.empty((H, S, D), dtype=np.uint16)
+    _check(lib().oracle_tapa_phase2(_p(p1), _p(head), P, S, H, D), "tapa_phase2")
+    return head
+
+
 def vmajor_metric(prev_v, cur_v, P, T):
     prev_v, cur_v = _u16(prev_v), _u16(cur_v)
     S, H, D = cur_v.shape

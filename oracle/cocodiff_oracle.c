@@ -11,6 +11,7 @@
  *     inverse (the second all-to-all of the same section);
  *   - QK normalisation (RMSNorm) and rotary embeddings on Q and K, never on V
  *     (Section II-B, "QK normalization" and "Rotary position embeddings");
+ *   - the two phases of the tile-aware parallel all-to-all (Section III-B);
  *   - the V-Major rule (Section III-D, "Active projection selection"): an L1
  *     distance between the current and the cached value vectors, the fraction
  *     r with the smallest distances is cached, the rest is active;
@@ -37,7 +38,8 @@
  *
  * Parity pins (tests/test_oracle_*.py, none of them re-types these formulas):
  * exchange - closed form HEAD[h][s] = SEQ[s][h] for every P, bijection, index
- * fill, sizes printed in the paper; norm - unit RMS, power-of-two scale
+ * fill, sizes printed in the paper; TAPA - each tile holds its GPU's tokens, the
+ * two phases compose to the flat exchange, rings are independent; norm - unit RMS, power-of-two scale
  * invariance, 3-4-5 hand case, fp64 textbook evaluation; RoPE - identity at
  * position 0, pair-norm preservation, relative-position property, quarter
  * turn, axis separation, complex-multiplication form; metric - brute force,
@@ -230,6 +232,62 @@ int oracle_ulysses_a2a_inverse(const uint16_t *head, uint16_t *seq, int P, int S
                 }
     free(sendbuf);
     free(recvbuf);
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Tile-aware parallel all-to-all (TAPA, Section III-B).  Ranks 2g and 2g+1    */
+/* are the two tiles of GPU g; P must be even.                                 */
+/* Phase 1: inside every GPU the two tiles swap their whole shards (S/P tokens,*/
+/* all heads - the "14 MB message" of the running example for Q, K, V), so     */
+/* that afterwards each tile holds all tokens of its GPU in token order.       */
+/* p1 layout: [2][P/2][2*S/P][H][D], p1[t][g] = what tile t of GPU g holds.    */
+/* With this layout p1[t] as a whole is again a [S][H][D] tensor.              */
+int oracle_tapa_phase1(const uint16_t *seq, uint16_t *p1, int P, int S, int H, int D) {
+    if (!shapes_ok(P, S, H, D) || P % 2 != 0) return ORACLE_BAD;
+    const int Sl = S / P, G = P / 2;
+    const size_t shard = (size_t)Sl * H * D; /* elements one tile owns and sends */
+    uint16_t *message = (uint16_t *)malloc(2 * (shard ? shard : 1));
+    if (!message) return ORACLE_BAD;
+    for (int g = 0; g < G; ++g)
+        for (int t = 0; t < 2; ++t) {
+            const int me = 2 * g + t, partner = 2 * g + (1 - t);
+            uint16_t *held = p1 + ((size_t)t * G + g) * 2 * shard; /* [2*Sl][H][D] */
+            /* own shard stays, at the position of tile t */
+            memcpy(held + (size_t)t * shard, seq + (size_t)me * shard, 2 * shard);
+            /* the partner's shard arrives as one message */
+            memcpy(message, seq + (size_t)partner * shard, 2 * shard);
+            memcpy(held + (size_t)(1 - t) * shard, message, 2 * shard);
+        }
+    free(message);
+    return ORACLE_OK;
+}
+
+/* Phase 2: two independent all-to-alls among the P/2 tiles of each ring      */
+/* (ring t = tile t of every GPU), no traffic between the rings.  Tile (g,t)   */
+/* sends to tile (g2,t) the tokens of GPU g restricted to the heads of rank    */
+/* 2*g2+t; the receiver lays the messages out by source GPU.                   */
+int oracle_tapa_phase2(const uint16_t *p1, uint16_t *head, int P, int S, int H, int D) {
+    if (!shapes_ok(P, S, H, D) || P % 2 != 0) return ORACLE_BAD;
+    const int Sl = S / P, Hl = H / P, G = P / 2, Sg = 2 * Sl; /* Sg tokens per GPU */
+    const size_t msg = (size_t)Sg * Hl * D;
+    uint16_t *message = (uint16_t *)malloc(2 * (msg ? msg : 1));
+    if (!message) return ORACLE_BAD;
+    for (int t = 0; t < 2; ++t)
+        for (int g = 0; g < G; ++g)
+            for (int g2 = 0; g2 < G; ++g2) {
+                const uint16_t *held = p1 + ((size_t)t * G + g) * Sg * H * D;
+                const int dst = 2 * g2 + t;
+                for (int j = 0; j < Sg; ++j)
+                    for (int hl = 0; hl < Hl; ++hl)
+                        memcpy(message + ((size_t)j * Hl + hl) * D,
+                               held + ((size_t)j * H + (size_t)dst * Hl + hl) * D, 2 * (size_t)D);
+                for (int j = 0; j < Sg; ++j)
+                    for (int hl = 0; hl < Hl; ++hl)
+                        memcpy(head + (((size_t)dst * Hl + hl) * S + (size_t)g * Sg + j) * D,
+                               message + ((size_t)j * Hl + hl) * D, 2 * (size_t)D);
+            }
+    free(message);
     return ORACLE_OK;
 }
 

@@ -104,3 +104,48 @@ def test_sizes_printed_in_the_paper():
     assert synth.config("qwen768")["grid"][0] == g["grid_768"][2]
     assert synth.config("temporal")["grid"][0] == g["grid_1536"][2]
     assert synth.config("qwen2304")["grid"][0] == g["grid_2304"][2]
+
+
+# ------------------------------------------------- TAPA (Section III-B) -----
+@pytest.mark.parametrize("P,S,H,D", [(2, 8, 2, 4), (4, 16, 4, 8), (6, 24, 12, 4), (12, 48, 12, 8)])
+def test_tapa_phase1_every_tile_holds_its_gpus_tokens(P, S, H, D):
+    x = _rand_bits((S, H, D), 20)
+    p1 = oracle.tapa_phase1(x, P).reshape(2, P // 2, 2 * S // P, H, D)
+    Sg = 2 * S // P
+    for t in range(2):
+        for g in range(P // 2):
+            assert np.array_equal(p1[t, g], x[g * Sg:(g + 1) * Sg])
+    # so each ring's copies, taken together, are the whole sequence-parallel tensor again
+    assert np.array_equal(oracle.tapa_phase1(x, P)[0], x) and np.array_equal(oracle.tapa_phase1(x, P)[1], x)
+
+
+@pytest.mark.parametrize("P,S,H,D", [(2, 8, 2, 4), (4, 16, 4, 8), (6, 24, 12, 4), (12, 48, 24, 8)])
+def test_tapa_phases_compose_to_the_flat_exchange(P, S, H, D):
+    x = _rand_bits((S, H, D), 21)
+    got = oracle.tapa_phase2(oracle.tapa_phase1(x, P), P)
+    assert np.array_equal(got, x.transpose(1, 0, 2))
+    assert np.array_equal(got, oracle.ulysses_a2a(x, P))
+
+
+def test_tapa_rings_are_independent():
+    """Phase 2 runs one all-to-all per ring with no traffic between them:
+    ranks of ring 0 depend only on the copies held by ring 0."""
+    P, S, H, D = 4, 16, 8, 4
+    x = _rand_bits((S, H, D), 22)
+    p1 = oracle.tapa_phase1(x, P)
+    base = oracle.tapa_phase2(p1, P).reshape(P, H // P, S, D)
+    p1b = p1.copy()
+    p1b[1] ^= np.uint16(0xFFFF)                       # corrupt everything ring 1 holds
+    got = oracle.tapa_phase2(p1b, P).reshape(P, H // P, S, D)
+    for r in range(P):
+        same = np.array_equal(got[r], base[r])
+        assert same == (r % 2 == 0), r
+
+
+def test_tapa_needs_an_even_rank_count_and_its_message_is_the_whole_shard():
+    with pytest.raises(ValueError):
+        oracle.tapa_phase1(_rand_bits((9, 3, 4), 23), 3)
+    g = _golden()
+    P, S, H, D = map(int, g["phase1_message_mb"][0].split())
+    # a tile sends its S/P tokens with all heads, for Q, K and V: "each message is 14 MB"
+    assert round(3 * (S // P) * H * D * 2 / 1e6) == g["phase1_message_mb"][2]
