@@ -195,6 +195,28 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
                                 void *workspace, size_t workspace_bytes, cocodiff_order order,
                                 void *stream_qk, void *stream_v);
 
+/* Tile-aware parallel all-to-all on virtual ranks (Section III-B, TAPA): ranks 2g
+ * and 2g+1 are the two tiles of GPU g; P must be even.  The two phases compose to
+ * cocodiff_ulysses_a2a bit for bit; they exist to reproduce the paper's data flow
+ * (what each tile holds after Phase 1, which the per-GPU selection scope works
+ * on), not to be faster: inside one device - and inside one NVLink domain -
+ * there is no bandwidth hierarchy to align to.
+ *
+ * Phase 1 (intra-GPU): the two tiles of a GPU swap their whole shards, so each
+ * tile holds all tokens of its GPU.  x_p1 = [2][P/2][2*S/P][H][D], x_p1[t][g] =
+ * holdings of tile t of GPU g (2*S*H*D elements per tensor); x_p1[t] as a whole
+ * is a [S][H][D] tensor, so V's x_p1[0] can be given directly to the V-Major
+ * calls (n_groups = P/2 is the per-GPU scope of the paper).
+ * Phase 2 (inter-GPU): one all-to-all per ring t (tile t of every GPU), no
+ * traffic between rings: rank 2*g2+t takes its heads from x_p1[t] only.
+ * Any (in, out) pair may be NULL/NULL. */
+int cocodiff_tapa_phase1(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                         uint16_t *q_p1, uint16_t *k_p1, uint16_t *v_p1,
+                         int P, int S, int H, int D, void *stream);
+int cocodiff_tapa_phase2(const uint16_t *q_p1, const uint16_t *k_p1, const uint16_t *v_p1,
+                         uint16_t *q_head, uint16_t *k_head, uint16_t *v_head,
+                         int P, int S, int H, int D, void *stream);
+
 /* cocodiff_vmajor_select_compact for callers that cannot allocate device memory.
  * (The paper has no counterpart: this is a deployment convenience of this library.)
  *

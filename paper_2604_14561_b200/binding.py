@@ -42,6 +42,8 @@ SIGNATURES = {
     "cocodiff_pack_active_qkv": (_I, [_P] * 5 + [_F] + [_P] * 6 + [_I] * 5 + [_P]),
     "cocodiff_unpack_qkv": (_I, [_P] * 8 + [_I] * 5 + [_P]),
     "cocodiff_vmajor_select_compact_static": (_I, [_P, _P] + [_I] * 5 + [_D, _I] + [_P] * 5 + [_P]),
+    "cocodiff_tapa_phase1": (_I, [_P] * 6 + [_I] * 4 + [_P]),
+    "cocodiff_tapa_phase2": (_I, [_P] * 6 + [_I] * 4 + [_P]),
     "cocodiff_selective_prologue": (_I, [_P] * 6 + [_F, _P] + [_I] * 5 + [_D, _I] + [_P] * 11 + [_Z, _I, _P, _P]),
 }
 
@@ -201,3 +203,13 @@ def vmajor_select_compact_static(prev_v, cur_v, P, S, H, D, T, r, n_groups, metr
     return _call("cocodiff_vmajor_select_compact_static", _ptr(prev_v), _ptr(cur_v), P, S, H, D, T, r,
                  n_groups, _ptr(metric), _ptr(mask), _ptr(idx), _ptr(n_active), _ptr(v_compact),
                  _stream(stream), check=check)
+
+
+def tapa_phase1(q, k, v, q_p1, k_p1, v_p1, P, S, H, D, stream=None, check=True):
+    return _call("cocodiff_tapa_phase1", _ptr(q), _ptr(k), _ptr(v), _ptr(q_p1), _ptr(k_p1), _ptr(v_p1),
+                 P, S, H, D, _stream(stream), check=check)
+
+
+def tapa_phase2(q_p1, k_p1, v_p1, q_head, k_head, v_head, P, S, H, D, stream=None, check=True):
+    return _call("cocodiff_tapa_phase2", _ptr(q_p1), _ptr(k_p1), _ptr(v_p1), _ptr(q_head), _ptr(k_head),
+                 _ptr(v_head), P, S, H, D, _stream(stream), check=check)

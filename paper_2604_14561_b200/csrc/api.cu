@@ -590,6 +590,71 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
     return COCODIFF_OK;
 }
 
+int cocodiff_tapa_phase1(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *q_p1,
+                         uint16_t *k_p1, uint16_t *v_p1, int P, int S, int H, int D, void *stream) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    if (P % 2 != 0) return COCODIFF_BAD_SHAPE;
+    const size_t E = (size_t)S * H * D, bytes = E * 2;
+    const uint16_t *in[3] = {q, k, v};
+    uint16_t *out[3] = {q_p1, k_p1, v_p1};
+    for (int i = 0; i < 3; ++i) {
+        if ((in[i] == nullptr) != (out[i] == nullptr)) return COCODIFF_INVALID_ARG;
+        if (!aligned16(in[i]) || !aligned16(out[i])) return COCODIFF_MISALIGNED;
+    }
+    for (int i = 0; i < 3; ++i)
+        for (int j = 0; j < 3; ++j) {
+            if (overlap(in[i], bytes, out[j], 2 * bytes)) return COCODIFF_ALIASING;
+            if (i < j && overlap(out[i], 2 * bytes, out[j], 2 * bytes)) return COCODIFF_ALIASING;
+        }
+    // The holdings of ring t, p1[t], are a [S][H][D] tensor: tile t keeps its own shard
+    // and receives its partner's.  On one device both are plain row copies.
+    for (int t = 0; t < 2; ++t) {
+        MoveParams p;
+        std::memset(&p, 0, sizeof p);
+        p.n_slots = S;
+        p.H = H;
+        p.src_tok = p.dst_tok = (long long)H * D;
+        p.src_head = p.dst_head = D;
+        p.map = MAP_FULL;
+        p.T = 1;
+        for (int i = 2; i >= 0; --i)
+            if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i] + (size_t)t * E, nullptr};
+        if (p.njobs == 0) return COCODIFF_OK;
+        CK(launch_move(p, D, (cudaStream_t)stream));
+    }
+    return COCODIFF_OK;
+}
+
+int cocodiff_tapa_phase2(const uint16_t *q_p1, const uint16_t *k_p1, const uint16_t *v_p1, uint16_t *q_head,
+                         uint16_t *k_head, uint16_t *v_head, int P, int S, int H, int D, void *stream) {
+    int rc = check_shape(P, S, H, D);
+    if (rc) return rc;
+    if (P % 2 != 0) return COCODIFF_BAD_SHAPE;
+    const size_t bytes = (size_t)S * H * D * 2;
+    const uint16_t *in[3] = {q_p1, k_p1, v_p1};
+    uint16_t *out[3] = {q_head, k_head, v_head};
+    for (int i = 0; i < 3; ++i) {
+        if ((in[i] == nullptr) != (out[i] == nullptr)) return COCODIFF_INVALID_ARG;
+        if (!aligned16(in[i]) || !aligned16(out[i])) return COCODIFF_MISALIGNED;
+    }
+    for (int i = 0; i < 3; ++i)
+        for (int j = 0; j < 3; ++j) {
+            if (overlap(in[i], 2 * bytes, out[j], bytes)) return COCODIFF_ALIASING;
+            if (i < j && overlap(out[i], bytes, out[j], bytes)) return COCODIFF_ALIASING;
+        }
+    TapaParams tp;
+    std::memset(&tp, 0, sizeof tp);
+    for (int i = 2; i >= 0; --i)
+        if (in[i]) { tp.src[tp.n] = in[i]; tp.dst[tp.n] = out[i]; ++tp.n; }
+    tp.S = S;
+    tp.H = H;
+    tp.Hl = H / P;
+    tp.heads_per_block = 8;
+    CK(launch_tapa_phase2(tp, D, (cudaStream_t)stream));
+    return COCODIFF_OK;
+}
+
 // ---------------------------------------------------------------------------
 // Scratch that lives in the library image, for callers that cannot allocate.
 // One array per GPU that loads the library, held until the process exits.

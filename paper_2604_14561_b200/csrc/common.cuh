@@ -59,6 +59,17 @@ struct MetricParams {
     SelectParams sel;
 };
 
+// Phase 2 of the two-phase exchange: up to three tensors, src = [2][S][H][D] (the
+// copies held by ring 0 and ring 1), dst = [H][S][D].
+struct TapaParams {
+    const uint16_t *src[3];
+    uint16_t *dst[3];
+    int n;                 // tensors
+    int S, H, Hl;          // Hl = H / P heads per rank
+    int heads_per_block;
+};
+
+cudaError_t launch_tapa_phase2(const TapaParams &p, int D, cudaStream_t stream);
 cudaError_t launch_move(const MoveParams &p, int D, cudaStream_t stream);
 cudaError_t launch_rope_table(float *cs, const int32_t *pos, int S, int D, double theta, cudaStream_t stream);
 cudaError_t launch_select(const SelectParams &p, cudaStream_t stream);
