@@ -179,3 +179,11 @@ def prologue(q, k, v, wq, wk, eps, cs, P):
     _check(lib().oracle_prologue(_p(q), _p(k), _p(v), _p(_u16(wq)), _p(_u16(wk)), C.c_float(eps),
                                  _p(cs), P, S, H, D, _p(qh), _p(kh), _p(vh), _p(scratch)), "prologue")
     return qh, kh, vh
+
+
+def cache_schedule(step, total_steps, warmup, sync_interval):
+    """(full_exchange, r) of a denoising step."""
+    full, r = C.c_int(0), C.c_double(0.0)
+    _check(lib().oracle_cache_schedule(step, total_steps, warmup, sync_interval, C.byref(full), C.byref(r)),
+           "cache_schedule")
+    return bool(full.value), float(r.value)

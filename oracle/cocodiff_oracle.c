@@ -409,6 +409,30 @@ int oracle_unpack(const uint16_t *compact, const int32_t *idx, int n_active, uin
 }
 
 /* ------------------------------------------------------------------------ */
+/* Time-varying cache schedule (Section III-D, "Time-varying cache            */
+/* scheduling").  Steps are numbered from 0.  (i) warm-up: the first `warmup`  */
+/* steps run the full exchange; (ii) from the warm-up boundary on the cache    */
+/* ratio r grows linearly from 0 (step `warmup`) to 1 (last step); (iii) every */
+/* `sync_interval`-th step is a full exchange that resets the cache.           */
+/* Reading: the paper gives no formula for the line nor the phase of the       */
+/* periodic refresh; taken here as r = (t - w) / (T - 1 - w) and full steps    */
+/* at t % interval == 0.                                                       */
+int oracle_cache_schedule(int step, int total_steps, int warmup, int sync_interval,
+                          int *full_exchange, double *r) {
+    if (step < 0 || total_steps < 1 || step >= total_steps || warmup < 0 || sync_interval < 0) return ORACLE_BAD;
+    int full = step < warmup;
+    if (sync_interval > 0 && step % sync_interval == 0) full = 1;
+    double ratio = 0.0;
+    if (step >= warmup) {
+        const int span = total_steps - 1 - warmup;
+        ratio = span > 0 ? (double)(step - warmup) / (double)span : 0.0;
+    }
+    *full_exchange = full;
+    *r = full ? 0.0 : ratio;
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------ */
 /* The whole prologue of one layer, full exchange: V is exchanged first       */
 /* (Section III-C), then Q and K after norm + RoPE.  Values do not depend on  */
 /* the order of issue.  scratch must hold S*H*D uint16.                       */
