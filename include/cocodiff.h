@@ -195,6 +195,33 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
                                 void *workspace, size_t workspace_bytes, cocodiff_order order,
                                 void *stream_qk, void *stream_v);
 
+/* Time-varying cache schedule (Section III-D, "Time-varying cache scheduling"),
+ * host-only arithmetic, steps numbered from 0:
+ *   - the first `warmup` steps and every step with step % sync_interval == 0
+ *     (sync_interval > 0) are full exchanges: *full_exchange = 1, *r = 0;
+ *   - otherwise *full_exchange = 0 and the cache ratio grows linearly from 0 at
+ *     step `warmup` to 1 at the last step: *r = (step - warmup) / (total_steps - 1 - warmup).
+ * The paper's experiments use total_steps = 50, warmup = 5, sync_interval = 10.
+ * full_exchange and r are HOST pointers. */
+int cocodiff_cache_schedule(int step, int total_steps, int warmup, int sync_interval,
+                            int *full_exchange, double *r);
+
+/* One denoising step of one layer under that schedule: a full step runs
+ * cocodiff_prologue straight into the three caches (resetting them to the exact
+ * values of this step); a selective step runs cocodiff_selective_prologue with
+ * the scheduled r.  All arguments as in those two calls; the caches are
+ * required.  sent_elements (HOST pointer, may be NULL) receives the number of
+ * bf16 elements of Q, K, V that cross the exchange in this step. */
+int cocodiff_layer_step(int step, int total_steps, int warmup, int sync_interval,
+                        const uint16_t *prev_v, const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                        const uint16_t *wq, const uint16_t *wk, float eps, const float *cs,
+                        int P, int S, int H, int D, int T, int n_groups,
+                        uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
+                        uint16_t *q_compact, uint16_t *k_compact, uint16_t *v_compact,
+                        uint16_t *q_cache, uint16_t *k_cache, uint16_t *v_cache,
+                        void *workspace, size_t workspace_bytes, cocodiff_order order,
+                        void *stream_qk, void *stream_v, int64_t *sent_elements);
+
 /* Tile-aware parallel all-to-all on virtual ranks (Section III-B, TAPA): ranks 2g
  * and 2g+1 are the two tiles of GPU g; P must be even.  The two phases compose to
  * cocodiff_ulysses_a2a bit for bit; they exist to reproduce the paper's data flow

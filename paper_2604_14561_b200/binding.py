@@ -42,6 +42,8 @@ SIGNATURES = {
     "cocodiff_pack_active_qkv": (_I, [_P] * 5 + [_F] + [_P] * 6 + [_I] * 5 + [_P]),
     "cocodiff_unpack_qkv": (_I, [_P] * 8 + [_I] * 5 + [_P]),
     "cocodiff_vmajor_select_compact_static": (_I, [_P, _P] + [_I] * 5 + [_D, _I] + [_P] * 5 + [_P]),
+    "cocodiff_cache_schedule": (_I, [_I] * 4 + [_P, _P]),
+    "cocodiff_layer_step": (_I, [_I] * 4 + [_P] * 6 + [_F, _P] + [_I] * 6 + [_P] * 11 + [_Z, _I, _P, _P, _P]),
     "cocodiff_tapa_phase1": (_I, [_P] * 6 + [_I] * 4 + [_P]),
     "cocodiff_tapa_phase2": (_I, [_P] * 6 + [_I] * 4 + [_P]),
     "cocodiff_selective_prologue": (_I, [_P] * 6 + [_F, _P] + [_I] * 5 + [_D, _I] + [_P] * 11 + [_Z, _I, _P, _P]),
@@ -213,3 +215,24 @@ def tapa_phase1(q, k, v, q_p1, k_p1, v_p1, P, S, H, D, stream=None, check=True):
 def tapa_phase2(q_p1, k_p1, v_p1, q_head, k_head, v_head, P, S, H, D, stream=None, check=True):
     return _call("cocodiff_tapa_phase2", _ptr(q_p1), _ptr(k_p1), _ptr(v_p1), _ptr(q_head), _ptr(k_head),
                  _ptr(v_head), P, S, H, D, _stream(stream), check=check)
+
+
+def cache_schedule(step, total_steps, warmup, sync_interval):
+    """(full_exchange, r) of a denoising step; host-only."""
+    full, r = C.c_int(0), C.c_double(0.0)
+    _call("cocodiff_cache_schedule", step, total_steps, warmup, sync_interval,
+          C.cast(C.byref(full), C.c_void_p), C.cast(C.byref(r), C.c_void_p))
+    return bool(full.value), float(r.value)
+
+
+def layer_step(step, total_steps, warmup, sync_interval, prev_v, q, k, v, wq, wk, eps, cs, P, S, H, D, T,
+               n_groups, metric, mask, idx, n_active, q_compact, k_compact, v_compact, q_cache, k_cache,
+               v_cache, workspace, workspace_bytes, order=V_FIRST, stream_qk=None, stream_v=None, check=True):
+    """Returns (status, elements of Q, K, V that cross the exchange in this step)."""
+    sent = C.c_int64(0)
+    rc = _call("cocodiff_layer_step", step, total_steps, warmup, sync_interval, _ptr(prev_v), _ptr(q), _ptr(k),
+               _ptr(v), _ptr(wq), _ptr(wk), eps, _ptr(cs), P, S, H, D, T, n_groups, _ptr(metric), _ptr(mask),
+               _ptr(idx), _ptr(n_active), _ptr(q_compact), _ptr(k_compact), _ptr(v_compact), _ptr(q_cache),
+               _ptr(k_cache), _ptr(v_cache), _ptr(workspace), workspace_bytes, order, _stream(stream_qk),
+               _stream(stream_v), C.cast(C.byref(sent), C.c_void_p), check=check)
+    return rc, int(sent.value)

@@ -590,6 +590,48 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
     return COCODIFF_OK;
 }
 
+int cocodiff_cache_schedule(int step, int total_steps, int warmup, int sync_interval, int *full_exchange,
+                            double *r) {
+    if (!full_exchange || !r || total_steps < 1 || step < 0 || step >= total_steps || warmup < 0 ||
+        sync_interval < 0)
+        return COCODIFF_INVALID_ARG;
+    const bool refresh = sync_interval > 0 && step % sync_interval == 0;
+    const bool full = step < warmup || refresh;
+    const int span = total_steps - 1 - warmup;
+    *full_exchange = full ? 1 : 0;
+    *r = (full || span <= 0) ? 0.0 : (double)(step - warmup) / (double)span;
+    return COCODIFF_OK;
+}
+
+int cocodiff_layer_step(int step, int total_steps, int warmup, int sync_interval, const uint16_t *prev_v,
+                        const uint16_t *q, const uint16_t *k, const uint16_t *v, const uint16_t *wq,
+                        const uint16_t *wk, float eps, const float *cs, int P, int S, int H, int D, int T,
+                        int n_groups, uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
+                        uint16_t *q_compact, uint16_t *k_compact, uint16_t *v_compact, uint16_t *q_cache,
+                        uint16_t *k_cache, uint16_t *v_cache, void *workspace, size_t workspace_bytes,
+                        cocodiff_order order, void *stream_qk, void *stream_v, int64_t *sent_elements) {
+    int full = 0;
+    double r = 0.0;
+    int rc = cocodiff_cache_schedule(step, total_steps, warmup, sync_interval, &full, &r);
+    if (rc) return rc;
+    if (!q_cache || !k_cache || !v_cache) return COCODIFF_INVALID_ARG;
+    if (full) {
+        rc = cocodiff_prologue(q, k, v, q_cache, k_cache, v_cache, wq, wk, eps, cs, P, S, H, D, order, stream_qk,
+                               stream_v);
+        if (rc == COCODIFF_OK && sent_elements) *sent_elements = 3LL * S * H * D;
+        return rc;
+    }
+    rc = cocodiff_selective_prologue(prev_v, q, k, v, wq, wk, eps, cs, P, S, H, D, T, r, n_groups, metric, mask,
+                                     idx, n_active, q_compact, k_compact, v_compact, q_cache, k_cache, v_cache,
+                                     workspace, workspace_bytes, order, stream_qk, stream_v);
+    if (rc == COCODIFF_OK && sent_elements) {
+        const int n = S / T, g = n / n_groups;
+        const long long act = n - (long long)n_groups * (long long)std::floor(r * (double)g);
+        *sent_elements = 3LL * act * T * H * D;
+    }
+    return rc;
+}
+
 int cocodiff_tapa_phase1(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *q_p1,
                          uint16_t *k_p1, uint16_t *v_p1, int P, int S, int H, int D, void *stream) {
     int rc = check_shape(P, S, H, D);

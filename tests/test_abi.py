@@ -102,3 +102,13 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", binding.LIB_PATH + ".absent")
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         binding.lib()
+
+
+def test_cache_schedule_matches_oracle_everywhere():
+    """Host-only entry point: compared with the oracle over a grid of settings."""
+    import oracle
+    for total, warmup, interval in ((50, 5, 10), (8, 1, 0), (20, 3, 5), (4, 0, 0), (6, 6, 0), (1, 0, 0), (30, 2, 7)):
+        for t in range(total):
+            assert binding.cache_schedule(t, total, warmup, interval) == oracle.cache_schedule(t, total, warmup, interval)
+    with pytest.raises(binding.CocodiffError):
+        binding.cache_schedule(5, 5, 0, 0)
