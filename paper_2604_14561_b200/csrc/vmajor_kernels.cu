@@ -21,11 +21,10 @@ constexpr int kCountMax = 512;  // groups up to this size are ranked by counting
 
 struct SelectSmem {
     int warp_sums[33];
-    int hist[256];
     int sel_bin, sel_k;
     unsigned long long mstar;
     int t_c;
-    unsigned long long stage[kCountMax];
+    unsigned long long stage[kCountMax];  // small groups: the metrics; also reduction slots
 };
 
 // Exclusive prefix sum of v over the block; *total receives the block sum.
@@ -58,87 +57,154 @@ __device__ __forceinline__ int block_excl_scan(int v, int *total, int *warp_sums
     return excl;
 }
 
-// Selection inside one group, by the whole block.
+// Block-wide maximum of a 64-bit value.
 template <int BLOCK>
-__device__ void select_group(const SelectParams &p, int grp, SelectSmem &sm) {
+__device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v, unsigned long long *slots) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, v, off);
+        v = o > v ? o : v;
+    }
+    if (lane == 0) slots[warp] = v;
+    __syncthreads();
+    unsigned long long r = slots[0];
+    for (int w = 1; w < BLOCK / 32; ++w) r = slots[w] > r ? slots[w] : r;
+    __syncthreads();
+    return r;
+}
+
+// Threshold form of the rule: with mstar the metric of the unit of rank
+// n_cached-1 in the order (metric, index), unit e is cached iff vals[e] < mstar,
+// or vals[e] == mstar and fewer than t_c units equal to mstar precede it.
+// Every thread owns a contiguous run of units, so two block scans suffice to
+// emit the mask and the ascending list.  vals may live in shared or global memory.
+template <int BLOCK>
+__device__ void emit_selection(const SelectParams &p, int grp, const unsigned long long *vals, bool none,
+                               unsigned long long mstar, int t_c, int *warp_sums) {
     const int tid = threadIdx.x;
-    const int g = p.g, base = grp * g, n_cached = p.n_cached;
-    const int out_base = grp * (g - n_cached);
-    const unsigned long long *m = p.metric + base;
-    const bool none = n_cached == 0;
-
-    // Threshold form of the rule: unit e is cached iff m[e] < mstar, or
-    // m[e] == mstar and fewer than t_c equal units precede it.
-    if (!none) {
-        if (g <= kCountMax) {
-            for (int e = tid; e < g; e += BLOCK) sm.stage[e] = m[e];
-            __syncthreads();
-            for (int e = tid; e < g; e += BLOCK) {
-                const unsigned long long my = sm.stage[e];
-                int less = 0, tie_before = 0;
-                for (int j = 0; j < g; ++j) {
-                    const unsigned long long o = sm.stage[j];
-                    less += o < my;
-                    tie_before += (o == my) & (j < e);
-                }
-                if (less + tie_before == n_cached - 1) { sm.mstar = my; sm.t_c = tie_before + 1; }
-            }
-            __syncthreads();
-        } else {
-            // radix select of the (n_cached-1)-th smallest metric, 8 bits per pass
-            unsigned long long prefix = 0, pmask = 0;
-            int k = n_cached - 1;
-            for (int shift = 56; shift >= 0; shift -= 8) {
-                for (int i = tid; i < 256; i += BLOCK) sm.hist[i] = 0;
-                __syncthreads();
-                for (int e = tid; e < g; e += BLOCK) {
-                    const unsigned long long v = m[e];
-                    if ((v & pmask) == prefix) atomicAdd(&sm.hist[(int)((v >> shift) & 255ull)], 1);
-                }
-                __syncthreads();
-                const int c = tid < 256 ? sm.hist[tid] : 0;
-                int total;
-                const int excl = block_excl_scan<BLOCK>(c, &total, sm.warp_sums);
-                if (tid < 256 && c > 0 && excl <= k && k < excl + c) { sm.sel_bin = tid; sm.sel_k = k - excl; }
-                __syncthreads();
-                prefix |= (unsigned long long)sm.sel_bin << shift;
-                pmask |= 0xffull << shift;
-                k = sm.sel_k;
-                __syncthreads();
-            }
-            if (tid == 0) { sm.mstar = prefix; sm.t_c = k + 1; }
-            __syncthreads();
+    const int g = p.g, base = grp * g, out_base = grp * (g - p.n_cached);
+    const int per = (g + BLOCK - 1) / BLOCK;
+    const int e_lo = tid * per < g ? tid * per : g;
+    const int e_hi = e_lo + per < g ? e_lo + per : g;
+    int ties = 0;
+    if (!none)
+        for (int e = e_lo; e < e_hi; ++e) ties += vals[e] == mstar;
+    int scan_total;
+    int tie_rank = block_excl_scan<BLOCK>(ties, &scan_total, warp_sums);
+    int actives = 0;
+    {
+        int tr = tie_rank;
+        for (int e = e_lo; e < e_hi; ++e) {
+            const unsigned long long v = vals[e];
+            const bool tie = !none && v == mstar;
+            const bool cached = !none && (v < mstar || (tie && tr < t_c));
+            tr += tie;
+            actives += !cached;
         }
     }
-    const unsigned long long mstar = none ? 0ull : sm.mstar;
-    const int t_c = none ? 0 : sm.t_c;
-
-    int tie_carry = 0, act_carry = 0;
-    for (int c0 = 0; c0 < g; c0 += BLOCK) {
-        const int e = c0 + tid;
-        const bool valid = e < g;
-        const unsigned long long v = valid ? m[e] : 0ull;
-        const int tie = (valid && !none && v == mstar) ? 1 : 0;
-        int tie_total, act_total;
-        const int tie_rank = tie_carry + block_excl_scan<BLOCK>(tie, &tie_total, sm.warp_sums);
-        const bool cached = valid && !none && (v < mstar || (tie && tie_rank < t_c));
-        const int active = (valid && !cached) ? 1 : 0;
-        const int pos = act_carry + block_excl_scan<BLOCK>(active, &act_total, sm.warp_sums);
-        if (valid) {
-            p.mask[base + e] = (uint8_t)active;
-            if (active) p.idx[out_base + pos] = base + e;
-        }
-        tie_carry += tie_total;
-        act_carry += act_total;
+    int pos = block_excl_scan<BLOCK>(actives, &scan_total, warp_sums);
+    for (int e = e_lo; e < e_hi; ++e) {
+        const unsigned long long v = vals[e];
+        const bool tie = !none && v == mstar;
+        const bool cached = !none && (v < mstar || (tie && tie_rank < t_c));
+        tie_rank += tie;
+        p.mask[base + e] = cached ? 0 : 1;
+        if (!cached) p.idx[out_base + pos++] = base + e;
     }
-    if (grp == 0 && tid == 0) *p.n_active = p.n_groups * (g - n_cached);
+    if (grp == 0 && tid == 0) *p.n_active = p.n_groups * (g - p.n_cached);
     __syncthreads();
 }
 
+// Small group (g <= kCountMax): every unit is ranked by counting in shared memory.
 template <int BLOCK>
-__global__ void __launch_bounds__(BLOCK) vmajor_select_kernel(const __grid_constant__ SelectParams p) {
+__device__ void select_group_small(const SelectParams &p, int grp, SelectSmem &sm) {
+    const int tid = threadIdx.x;
+    const int g = p.g, n_cached = p.n_cached;
+    const unsigned long long *m = p.metric + (long long)grp * g;
+    const bool none = n_cached == 0;
+    for (int e = tid; e < g; e += BLOCK) sm.stage[e] = m[e];
+    __syncthreads();
+    if (!none) {
+        for (int e = tid; e < g; e += BLOCK) {
+            const unsigned long long my = sm.stage[e];
+            int less = 0, tie_before = 0;
+            for (int j = 0; j < g; ++j) {
+                const unsigned long long o = sm.stage[j];
+                less += o < my;
+                tie_before += (o == my) & (j < e);
+            }
+            if (less + tie_before == n_cached - 1) { sm.mstar = my; sm.t_c = tie_before + 1; }
+        }
+        __syncthreads();
+    }
+    emit_selection<BLOCK>(p, grp, sm.stage, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm.warp_sums);
+}
+
+// Large group: radix select (8 bits per pass, starting at the highest byte in
+// use) of the metric of rank n_cached-1.  The metrics are staged in dynamic
+// shared memory when they fit (staged != 0); every warp keeps its own histogram
+// so that clustered metrics do not serialise the whole block on one counter.
+template <int BLOCK>
+__device__ void select_group_large(const SelectParams &p, int grp, SelectSmem &sm, unsigned long long *dyn_vals,
+                                   int *warp_hist, int staged) {
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int g = p.g, n_cached = p.n_cached;
+    const unsigned long long *m = p.metric + (long long)grp * g;
+    const bool none = n_cached == 0;
+    const unsigned long long *vals = m;
+    unsigned long long mx = 0;
+    for (int e = tid; e < g; e += BLOCK) {
+        const unsigned long long v = m[e];
+        if (staged) dyn_vals[e] = v;
+        mx = v > mx ? v : mx;
+    }
+    if (staged) vals = dyn_vals;
+    mx = block_max_u64<BLOCK>(mx, sm.stage);  // also publishes the staged values
+    if (!none) {
+        int top = 56;
+        while (top > 0 && (mx >> top) == 0ull) top -= 8;
+        unsigned long long prefix = 0, pmask = 0;
+        int k = n_cached - 1;
+        int *my_hist = warp_hist + warp * 256;
+        for (int shift = top; shift >= 0; shift -= 8) {
+            for (int i = tid; i < (BLOCK / 32) * 256; i += BLOCK) warp_hist[i] = 0;
+            __syncthreads();
+            for (int e = tid; e < g; e += BLOCK) {
+                const unsigned long long v = vals[e];
+                if ((v & pmask) == prefix) atomicAdd(&my_hist[(int)((v >> shift) & 255ull)], 1);
+            }
+            __syncthreads();
+            int c = 0;
+            if (tid < 256)
+                for (int w = 0; w < BLOCK / 32; ++w) c += warp_hist[w * 256 + tid];
+            int total;
+            const int excl = block_excl_scan<BLOCK>(c, &total, sm.warp_sums);
+            if (tid < 256 && c > 0 && excl <= k && k < excl + c) { sm.sel_bin = tid; sm.sel_k = k - excl; }
+            __syncthreads();
+            prefix |= (unsigned long long)sm.sel_bin << shift;
+            pmask |= 0xffull << shift;
+            k = sm.sel_k;
+            __syncthreads();
+        }
+        if (tid == 0) { sm.mstar = prefix; sm.t_c = k + 1; }
+        __syncthreads();
+    }
+    emit_selection<BLOCK>(p, grp, vals, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm.warp_sums);
+}
+
+__global__ void __launch_bounds__(256) vmajor_select_small_kernel(const __grid_constant__ SelectParams p) {
     __shared__ SelectSmem sm;
-    select_group<BLOCK>(p, blockIdx.x, sm);
+    select_group_small<256>(p, blockIdx.x, sm);
+}
+
+constexpr int kLargeBlock = 1024;
+__global__ void __launch_bounds__(kLargeBlock)
+vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int staged) {
+    __shared__ SelectSmem sm;
+    __shared__ int warp_hist[(kLargeBlock / 32) * 256];
+    extern __shared__ unsigned long long dyn_vals[];
+    select_group_large<kLargeBlock>(p, blockIdx.x, sm, dyn_vals, warp_hist, staged);
 }
 
 // fix(|a - b|): one fp32 subtraction, scale by 2^16, truncate, saturate to 32
@@ -204,19 +270,32 @@ vmajor_metric_kernel(const __grid_constant__ MetricParams p, const int fuse_sele
     for (int u = threadIdx.x; u < p.n_units; u += kMetricThreads) p.metric[u] = __ldcg(p.acc + u);
     __syncthreads();
     if (fuse_select)
-        for (int grp = 0; grp < p.sel.n_groups; ++grp) select_group<kMetricThreads>(p.sel, grp, sm);
+        for (int grp = 0; grp < p.sel.n_groups; ++grp) select_group_small<kMetricThreads>(p.sel, grp, sm);
 }
 
 }  // namespace
 
 cudaError_t launch_select(const SelectParams &p, cudaStream_t stream) {
-    if (p.n == 0) {
-        return cudaMemsetAsync(p.n_active, 0, sizeof(int32_t), stream);
+    if (p.n == 0) return cudaMemsetAsync(p.n_active, 0, sizeof(int32_t), stream);
+    if (p.g <= kCountMax) {
+        vmajor_select_small_kernel<<<p.n_groups, 256, 0, stream>>>(p);
+        return cudaGetLastError();
     }
-    if (p.g <= kCountMax)
-        vmajor_select_kernel<256><<<p.n_groups, 256, 0, stream>>>(p);
-    else
-        vmajor_select_kernel<1024><<<p.n_groups, 1024, 0, stream>>>(p);
+    // stage the group's metrics in shared memory when they fit beside the histograms
+    const size_t want = (size_t)p.g * sizeof(unsigned long long);
+    const size_t limit = 160 * 1024;
+    const int staged = want <= limit ? 1 : 0;
+    const size_t dyn = staged ? want : 0;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        e = cudaFuncSetAttribute(vmajor_select_large_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    vmajor_select_large_kernel<<<p.n_groups, kLargeBlock, dyn, stream>>>(p, staged);
     return cudaGetLastError();
 }
 
@@ -230,7 +309,9 @@ cudaError_t launch_metric_select(const MetricParams &p, cudaStream_t stream) {
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const long long cap = (long long)sms * 4;
     if (blocks > cap) blocks = cap;
-    const int fuse = (p.sel.g <= kCountMax && p.sel.n_groups <= 64) ? 1 : 0;
+    // one small group: its selection rides in the metric kernel's last block; several
+    // groups or a large one go to their own launch, one block per group
+    const int fuse = (p.sel.g <= kCountMax && p.sel.n_groups <= 2) ? 1 : 0;
     vmajor_metric_kernel<<<(unsigned)blocks, kMetricThreads, 0, stream>>>(p, fuse);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || fuse) return e;
