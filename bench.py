@@ -185,6 +185,32 @@ def time_loop(torch, fn, stream, steps, warmup=3):
     return a.elapsed_time(b) / steps
 
 
+def time_graph(torch, fn, stream, steps, flush=None):
+    """Capture one call of `fn` (already warmed up) into a CUDA graph on `stream`
+    and time its replays; returns per-replay ms, or None if capture is refused."""
+    try:
+        g = torch.cuda.CUDAGraph()
+        stream.synchronize()
+        torch.cuda.synchronize()
+        with torch.cuda.graph(g, stream=stream):
+            fn()
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        with torch.cuda.stream(stream):
+            for a, b in ev:
+                if flush is not None:
+                    flush()
+                a.record(stream)
+                g.replay()
+                b.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in ev]
+    except Exception as exc:                      # capture not possible: report, do not fail the bench
+        sys.stderr.write(f"graph capture skipped: {exc}\n")
+        return None
+
+
 def max_over_ranks(ms, world, device):
     """The slowest rank's time: every multi-GPU number is the max over ranks."""
     if world <= 1:
@@ -390,6 +416,9 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
             warm = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 3))
             out[name][oname] = {"us_cold_l2": 1e3 * cold, "gbs_cold_l2": b / (cold * 1e-3) / 1e9,
                                 "us_warm_l2": 1e3 * warm}
+            gr = time_graph(torch, lambda: full(order), sq, iters, flush=flush)
+            if gr is not None:
+                out[name][oname]["us_cold_l2_cuda_graph"] = 1e3 * statistics.median(gr)
         if name != "temporal":
             continue
         # selective step: metric + selection + V compaction, K/Q compaction (norm + RoPE fused), three scatters
@@ -416,6 +445,9 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
         for oname, order in (("lump", binding.LUMP), ("v_first", binding.V_FIRST)):
             cold = time_steps(torch, lambda: selective(order), sq, iters, 3, flush=flush)
             sel[oname] = 1e3 * statistics.median(cold)
+            gr = time_graph(torch, lambda: selective(order), sq, iters, flush=flush)
+            if gr is not None:
+                sel[oname + "_cuda_graph"] = 1e3 * statistics.median(gr)
         n_act = int(na.item())
         tile = T * H * D * 2
         sb = 2 * E * 2 + 3 * 2 * n_act * tile + 3 * 2 * n_act * tile

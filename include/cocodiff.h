@@ -105,9 +105,11 @@ int cocodiff_prologue(const uint16_t *q, const uint16_t *k, const uint16_t *v,
 
 /* The same prologue for HOST tensors: q, k, v and the three results are host
  * pointers (pinned memory makes the copies asynchronous); dev_in and dev_out
- * are caller-owned device staging buffers of 3*S*H*D bf16 each.  V is copied,
- * exchanged and copied back on stream_v while Q and K follow on stream_qk
- * (V_FIRST), or everything runs on stream_qk (LUMP).  wq, wk, cs stay device
+ * are caller-owned device staging buffers of 3*S*H*D bf16 each.  With V_FIRST
+ * and two streams the tokens are processed in chunks that alternate between
+ * the streams, so that host-to-device copies, the kernel and device-to-host
+ * copies of neighbouring chunks overlap; inside a chunk V leads.  With LUMP (or
+ * equal streams) everything runs in order on stream_qk.  wq, wk, cs stay device
  * pointers.  On return stream_qk is ordered after all of it. */
 int cocodiff_prologue_host(const uint16_t *q_host, const uint16_t *k_host, const uint16_t *v_host,
                            uint16_t *q_head_host, uint16_t *k_head_host, uint16_t *v_head_host,

@@ -19,7 +19,7 @@
  *     "Selective communication in TAPA") and the receiver-side indexed scatter
  *     over the cached head-parallel tensors ("Post-Phase 2").
  *
- * Readings where the paper gives no formula (all listed in the design notes):
+ * Readings taken where the paper gives no formula:
  *   - RMSNorm is per (token, head) over the D head dimensions, eps inside the
  *     square root, one bf16 weight vector [D] per tensor.
  *   - RoPE is axial 2-D: the first D/2 dimensions rotate with the row position,

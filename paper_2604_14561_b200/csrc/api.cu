@@ -377,11 +377,11 @@ int cocodiff_prologue_host(const uint16_t *q_host, const uint16_t *k_host, const
     if (overlap(dev_in, 3 * bytes, dev_out, 3 * bytes)) return COCODIFF_ALIASING;
     cudaStream_t sq = (cudaStream_t)stream_qk, sv = (cudaStream_t)stream_v;
     if (order == COCODIFF_LUMP) sv = sq;
-    uint16_t *dq = dev_in, *dk = dev_in + E, *dv = dev_in + 2 * E;
-    uint16_t *oq = dev_out, *ok = dev_out + E, *ov = dev_out + 2 * E;
-    MoveParams base = seq_to_head(S, H, D);
-    base.cs = cs;
-    base.eps = eps;
+    uint16_t *din[3] = {dev_in + 2 * E, dev_in, dev_in + E};      // V, Q, K
+    uint16_t *dout[3] = {dev_out + 2 * E, dev_out, dev_out + E};
+    const uint16_t *hin[3] = {v_host, q_host, k_host};
+    uint16_t *hout[3] = {v_head_host, q_head_host, k_head_host};
+    const uint16_t *w[3] = {nullptr, wq, wk};
     ForkJoin *fj = nullptr;
     if (sv != sq) {
         rc = get_events(&fj);
@@ -389,20 +389,30 @@ int cocodiff_prologue_host(const uint16_t *q_host, const uint16_t *k_host, const
         CK(cudaEventRecord(fj->fork, sq));
         CK(cudaStreamWaitEvent(sv, fj->fork, 0));
     }
-    // V first: copy in, exchange, copy out on its own stream
-    CK(cudaMemcpyAsync(dv, v_host, bytes, cudaMemcpyHostToDevice, sv));
-    MoveParams pv = base;
-    pv.job[pv.njobs++] = MoveJob{dv, ov, nullptr};
-    CK(launch_move(pv, D, sv));
-    CK(cudaMemcpyAsync(v_head_host, ov, bytes, cudaMemcpyDeviceToHost, sv));
-    CK(cudaMemcpyAsync(dq, q_host, bytes, cudaMemcpyHostToDevice, sq));
-    CK(cudaMemcpyAsync(dk, k_host, bytes, cudaMemcpyHostToDevice, sq));
-    MoveParams pqk = base;
-    pqk.job[pqk.njobs++] = MoveJob{dq, oq, wq};
-    pqk.job[pqk.njobs++] = MoveJob{dk, ok, wk};
-    CK(launch_move(pqk, D, sq));
-    CK(cudaMemcpyAsync(q_head_host, oq, bytes, cudaMemcpyDeviceToHost, sq));
-    CK(cudaMemcpyAsync(k_head_host, ok, bytes, cudaMemcpyDeviceToHost, sq));
+    // Token chunks alternate between the two streams: while one chunk's results
+    // travel back to the host, the next chunk's inputs arrive and its rows are
+    // processed.  Inside a chunk V is copied first and its blocks lead the grid.
+    const int n_chunks = (sv != sq && S >= 8 * 256) ? 8 : 1;
+    int chunk = (S + n_chunks - 1) / n_chunks;
+    chunk = (chunk + 31) / 32 * 32;
+    const size_t tok_in = (size_t)H * D, pitch = (size_t)S * D * 2;
+    for (int c = 0, s0 = 0; s0 < S; ++c, s0 += chunk) {
+        const int len = s0 + chunk <= S ? chunk : S - s0;
+        cudaStream_t st = (c % 2 == 0) ? sv : sq;
+        MoveParams p = seq_to_head(S, H, D);
+        p.n_slots = len;
+        p.cs = cs + (size_t)s0 * D;
+        p.eps = eps;
+        for (int i = 0; i < 3; ++i) {
+            CK(cudaMemcpyAsync(din[i] + s0 * tok_in, hin[i] + s0 * tok_in, (size_t)len * tok_in * 2,
+                               cudaMemcpyHostToDevice, st));
+            p.job[p.njobs++] = MoveJob{din[i] + s0 * tok_in, dout[i] + (size_t)s0 * D, w[i]};
+        }
+        CK(launch_move(p, D, st));
+        for (int i = 0; i < 3; ++i)
+            CK(cudaMemcpy2DAsync(hout[i] + (size_t)s0 * D, pitch, dout[i] + (size_t)s0 * D, pitch,
+                                 (size_t)len * D * 2, (size_t)H, cudaMemcpyDeviceToHost, st));
+    }
     if (sv != sq) {
         CK(cudaEventRecord(fj->join, sv));
         CK(cudaStreamWaitEvent(sq, fj->join, 0));

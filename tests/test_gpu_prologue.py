@@ -136,8 +136,9 @@ def test_qk_norm_rope_alone_and_in_place(S, H, D):
     assert_norm_rope_close(ko.host((S, H, D)), ref, ref_f, "k norm only")
 
 
-def test_prologue_host_buffers_match_device_path():
-    cfg = synth.config("tiny")
+@pytest.mark.parametrize("name", ["tiny", "qwen768"])      # one chunk / eight pipelined token chunks
+def test_prologue_host_buffers_match_device_path(name):
+    cfg = synth.config(name)
     L = synth.make_layer(cfg)
     S, H, D, P = cfg["S"], cfg["H"], cfg["D"], cfg["P"]
     E = S * H * D
