@@ -157,3 +157,40 @@ def test_prologue_host_buffers_match_device_path(name):
         for got, ref in zip(hout, want):
             assert np.array_equal(got.numpy().view(np.uint16).reshape(H, S, D), ref)
             got.zero_()
+
+
+def test_exchange_and_norm_beyond_2_31_elements():
+    """One tensor of 2.4e9 elements (4.8 GB): offsets no longer fit 32 bits.
+    Checked on the device against what holds at any size: the exchange is the
+    axis swap HEAD[h][s] = SEQ[s][h], its inverse restores the input, and a
+    normalised row (weight 1, no rotation) has unit RMS."""
+    P, S, H, D = 16, 1179648, 16, 128
+    E = S * H * D
+    assert E > 2 ** 31
+    g = torch.Generator(device="cuda").manual_seed(0)
+    x = torch.empty(E, dtype=torch.int16, device="cuda")
+    for lo in range(0, E, 1 << 28):        # bf16 patterns of N(0,1) values, generated on the device
+        hi = min(E, lo + (1 << 28))
+        x[lo:hi] = torch.randn(hi - lo, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16).view(torch.int16)
+    y = torch.empty(E, dtype=torch.int16, device="cuda")
+    binding.ulysses_a2a(None, None, x, None, None, y, P, S, H, D, order=binding.LUMP)
+    torch.cuda.synchronize()
+    xv, yv = x.view(S, H, D), y.view(H, S, D)
+    for h in range(H):
+        assert torch.equal(yv[h], xv[:, h, :]), h
+    back = torch.empty(E, dtype=torch.int16, device="cuda")
+    binding.ulysses_a2a_inverse(None, None, y, None, None, back, P, S, H, D)
+    torch.cuda.synchronize()
+    assert torch.equal(back, x)
+    del back
+    w = torch.full((D,), 0x3F80, dtype=torch.int16, device="cuda")        # bf16 1.0
+    # normalisation only (no table): SEQ -> SEQ
+    binding.qk_norm_rope(x, None, y, None, w, None, 1e-6, None, S, H, D)
+    torch.cuda.synchronize()
+    rows = y.view(torch.bfloat16).view(S * H, D)
+    for lo in (0, S * H // 2 - 1000, S * H - 4096):                        # first, middle and last rows
+        r = rows[lo:lo + 4096].float()
+        rms = r.pow(2).mean(dim=1).sqrt()
+        assert torch.all((rms - 1.0).abs() < 2.0 ** -8), lo
+    # and the normalised rows are the right rows: same signs as the input rows they came from
+    assert torch.equal((y.view(S * H, D)[-4096:] < 0), (x.view(S * H, D)[-4096:] < 0))
