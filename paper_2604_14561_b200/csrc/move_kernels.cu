@@ -147,8 +147,11 @@ __global__ void __launch_bounds__(THREADS, MINB) move_rows_kernel(const __grid_c
     }
 
     // Per-token constants, reused for all heads: the norm weight folded into the
-    // rotation.  out[2q] = inv*(x[2q]*ka - x[2q+1]*kb), out[2q+1] = inv*(x[2q]*kc + x[2q+1]*kd).
-    float ka[4], kb[4], kc[4], kd[4];
+    // rotation.  With pair q = elements (2q, 2q+1) = (a_q, b_q):
+    //   out[2q] = inv * (a_q*ka_q + b_q*kb_q),  out[2q+1] = inv * (a_q*kc_q + b_q*kd_q).
+    // Pairs (0,1) and (2,3) are processed together with sm_100's packed fp32x2
+    // arithmetic (two independent IEEE fp32 operations per instruction).
+    float2 ka01, kb01, kc01, kd01, ka23, kb23, kc23, kd23;
     {
         float w[8];
         unpack8(__ldg(reinterpret_cast<const uint4 *>(job.w) + lr), w);
@@ -160,33 +163,36 @@ __global__ void __launch_bounds__(THREADS, MINB) move_rows_kernel(const __grid_c
             c[0] = t0.x; sn[0] = t0.y; c[1] = t0.z; sn[1] = t0.w;
             c[2] = t1.x; sn[2] = t1.y; c[3] = t1.z; sn[3] = t1.w;
         }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            ka[q] = w[2 * q] * c[q];
-            kb[q] = -(w[2 * q + 1] * sn[q]);
-            kc[q] = w[2 * q] * sn[q];
-            kd[q] = w[2 * q + 1] * c[q];
-        }
+        ka01 = make_float2(w[0] * c[0], w[2] * c[1]);
+        kb01 = make_float2(-(w[1] * sn[0]), -(w[3] * sn[1]));
+        kc01 = make_float2(w[0] * sn[0], w[2] * sn[1]);
+        kd01 = make_float2(w[1] * c[0], w[3] * c[1]);
+        ka23 = make_float2(w[4] * c[2], w[6] * c[3]);
+        kb23 = make_float2(-(w[5] * sn[2]), -(w[7] * sn[3]));
+        kc23 = make_float2(w[4] * sn[2], w[6] * sn[3]);
+        kd23 = make_float2(w[5] * c[2], w[7] * c[3]);
     }
     const float inv_d = 1.0f / (float)D;
     const float eps = p.eps;
 
     auto norm_rope_row = [&](const uint4 v) -> uint4 {
-        float x[8];
-        unpack8(v, x);
-        float ss = x[0] * x[0];
-#pragma unroll
-        for (int j = 1; j < 8; ++j) ss = fmaf(x[j], x[j], ss);
-        ss = group_sum<LPR>(ss);
+        // a_q = low bf16 of word q, b_q = high bf16 of word q, widened exactly
+        const float2 a01 = make_float2(__uint_as_float(v.x << 16), __uint_as_float(v.y << 16));
+        const float2 b01 = make_float2(__uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y & 0xffff0000u));
+        const float2 a23 = make_float2(__uint_as_float(v.z << 16), __uint_as_float(v.w << 16));
+        const float2 b23 = make_float2(__uint_as_float(v.z & 0xffff0000u), __uint_as_float(v.w & 0xffff0000u));
+        float2 acc = __fmul2_rn(a01, a01);
+        acc = __ffma2_rn(b01, b01, acc);
+        acc = __ffma2_rn(a23, a23, acc);
+        acc = __ffma2_rn(b23, b23, acc);
+        const float ss = group_sum<LPR>(acc.x + acc.y);
         const float inv = rsqrt_approx(fmaf(ss, inv_d, eps));
-        unsigned out[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const float lo = fmaf(x[2 * q], ka[q], x[2 * q + 1] * kb[q]) * inv;
-            const float hi = fmaf(x[2 * q], kc[q], x[2 * q + 1] * kd[q]) * inv;
-            out[q] = pack2(lo, hi);
-        }
-        return make_uint4(out[0], out[1], out[2], out[3]);
+        const float2 inv2 = make_float2(inv, inv);
+        const float2 lo01 = __fmul2_rn(__ffma2_rn(a01, ka01, __fmul2_rn(b01, kb01)), inv2);
+        const float2 hi01 = __fmul2_rn(__ffma2_rn(a01, kc01, __fmul2_rn(b01, kd01)), inv2);
+        const float2 lo23 = __fmul2_rn(__ffma2_rn(a23, ka23, __fmul2_rn(b23, kb23)), inv2);
+        const float2 hi23 = __fmul2_rn(__ffma2_rn(a23, kc23, __fmul2_rn(b23, kd23)), inv2);
+        return make_uint4(pack2(lo01.x, hi01.x), pack2(lo01.y, hi01.y), pack2(lo23.x, hi23.x), pack2(lo23.y, hi23.y));
     };
 
     int h = h_lo;
