@@ -168,7 +168,7 @@ int check_tiles(const uint16_t *const in[3], uint16_t *const out[3], int S, int 
 
 int enqueue_metric_select(const uint16_t *prev_v, const uint16_t *cur_v, int S, int H, int D, int T, double r,
                           int n_groups, uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
-                          void *workspace, cudaStream_t st) {
+                          void *workspace, cudaStream_t st, int pdl = 0) {
     const int n = S / T;
     const size_t need = vmajor_ws_bytes(S, T);
     MetricParams mp;
@@ -190,6 +190,7 @@ int enqueue_metric_select(const uint16_t *prev_v, const uint16_t *cur_v, int S, 
     mp.sel.mask = mask;
     mp.sel.idx = idx;
     mp.sel.n_active = n_active;
+    mp.pdl = pdl;
     CK(cudaMemsetAsync(workspace, 0, need, st));
     CK(launch_metric_select(mp, st));
     return COCODIFF_OK;
@@ -198,7 +199,7 @@ int enqueue_metric_select(const uint16_t *prev_v, const uint16_t *cur_v, int S, 
 // Compaction of up to three tensors in one launch; slot order (Q, K, V), V's blocks first.
 int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint16_t *wq, const uint16_t *wk,
                  float eps, const float *cs, const int32_t *idx, const int32_t *n_active, int slots, int S,
-                 int H, int D, int T, cudaStream_t st) {
+                 int H, int D, int T, cudaStream_t st, int pdl = 0) {
     (void)S;
     MoveParams p;
     std::memset(&p, 0, sizeof p);
@@ -210,6 +211,8 @@ int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint
     p.dst_head = COMPACT_STRIDE;
     p.map = MAP_GATHER;
     p.T = T;
+    p.n_units = S / T;
+    p.pdl = pdl;
     p.idx = idx;
     p.n_active = n_active;
     p.cs = cs;
@@ -223,7 +226,7 @@ int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint
 }
 
 int enqueue_unpack(const uint16_t *const in[3], uint16_t *const out[3], const int32_t *idx,
-                   const int32_t *n_active, int slots, int S, int H, int D, int T, cudaStream_t st) {
+                   const int32_t *n_active, int slots, int S, int H, int D, int T, cudaStream_t st, int pdl = 0) {
     MoveParams p;
     std::memset(&p, 0, sizeof p);
     p.n_slots = slots;
@@ -234,6 +237,8 @@ int enqueue_unpack(const uint16_t *const in[3], uint16_t *const out[3], const in
     p.dst_head = (long long)S * D;
     p.map = MAP_SCATTER;
     p.T = T;
+    p.n_units = S / T;
+    p.pdl = pdl;
     p.idx = idx;
     p.n_active = n_active;
     for (int i = 2; i >= 0; --i)
@@ -463,9 +468,12 @@ int cocodiff_vmajor_select_compact(const uint16_t *prev_v, const uint16_t *cur_v
         if (overlap(prev_v, (size_t)S * H * D * 2, v_compact, (size_t)S * H * D * 2)) return COCODIFF_ALIASING;
     }
     cudaStream_t st = (cudaStream_t)stream;
-    rc = enqueue_metric_select(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, st);
+    rc = enqueue_metric_select(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, st,
+                               v_compact ? PDL_TRIGGER : 0);
     if (rc) return rc;
-    if (v_compact) return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, S, S, H, D, T, st);
+    if (v_compact)
+        return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, S, S, H, D, T, st,
+                            PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
     return COCODIFF_OK;
 }
 
@@ -568,11 +576,18 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
     const int n = S / T, g = n / n_groups;
     const int slots = (n - n_groups * (int)std::floor(r * (double)g)) * T;
     cudaStream_t sq = (cudaStream_t)stream_qk, sv = (cudaStream_t)stream_v;
+    // On one stream the three kernels are chained with programmatic dependent launches:
+    // each successor becomes resident while its predecessor drains and orders itself
+    // with griddepcontrol.wait, which hides its launch latency and ramp-up.
+    int unpack_pdl = 0;
     if (order == COCODIFF_LUMP || sv == sq) {
-        rc = enqueue_metric_select(prev_v, v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, sq);
+        rc = enqueue_metric_select(prev_v, v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, sq,
+                                   PDL_TRIGGER);
         if (rc) return rc;
-        rc = enqueue_pack(in, comp, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T, sq);
+        rc = enqueue_pack(in, comp, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T, sq,
+                          PDL_LAUNCH_ATTR | PDL_WAIT_AT_START | PDL_TRIGGER);
         if (rc) return rc;
+        unpack_pdl = PDL_LAUNCH_ATTR | PDL_WAIT_AT_START;
     } else {
         // V first: metric, selection and V's compaction on stream_v; Q and K follow on
         // stream_qk as soon as the index list exists.
@@ -596,7 +611,7 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
         CK(cudaEventRecord(fj->join, sv));
         CK(cudaStreamWaitEvent(sq, fj->join, 0));
     }
-    if (do_unpack) return enqueue_unpack(comp_in, cache, idx, n_active, slots, S, H, D, T, sq);
+    if (do_unpack) return enqueue_unpack(comp_in, cache, idx, n_active, slots, S, H, D, T, sq, unpack_pdl);
     return COCODIFF_OK;
 }
 
@@ -755,9 +770,12 @@ int cocodiff_vmajor_select_compact_static(const uint16_t *prev_v, const uint16_t
     }
     cudaStream_t st = (cudaStream_t)stream;
     // enqueue_metric_select clears the accumulators and the ticket it is about to use
-    rc = enqueue_metric_select(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, scratch, st);
+    rc = enqueue_metric_select(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, scratch, st,
+                               v_compact ? PDL_TRIGGER : 0);
     if (rc) return rc;
-    if (v_compact) return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, S, S, H, D, T, st);
+    if (v_compact)
+        return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, S, S, H, D, T, st,
+                            PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
     return COCODIFF_OK;
 }
 

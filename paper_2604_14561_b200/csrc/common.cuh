@@ -12,6 +12,18 @@ enum TokenMap : int {
     MAP_SCATTER = 2   // src token = o, dst token = idx[o / T] * T + o % T  (reconstruction)
 };
 
+// Programmatic dependent launch (same-stream overlap of consecutive kernels).
+// A kernel launched with the programmatic attribute may start while its
+// predecessor in the stream is still running; it then orders itself with
+// griddepcontrol.wait, which returns once the predecessor has completed and its
+// writes are visible.  Without the launch attribute these instructions do nothing.
+enum PdlFlags : int {
+    PDL_WAIT_AT_START = 1,   // the kernel consumes its predecessor's results
+    PDL_TRIGGER = 2,         // let the successor start as soon as every block of this grid runs
+    PDL_WAIT_AT_END = 4,     // independent of the predecessor, but must not complete before it
+    PDL_LAUNCH_ATTR = 8      // host side: launch with programmatic stream serialization
+};
+
 struct MoveJob {
     const uint16_t *src;
     uint16_t *dst;
@@ -34,7 +46,9 @@ struct MoveParams {
     const int32_t *idx;     // active units (MAP_GATHER / MAP_SCATTER)
     const int32_t *n_active;
     int T;
+    int n_units;            // S / T: indices read from idx are clamped to [0, n_units)
     int map;
+    int pdl;                // programmatic dependent launch: see PdlFlags
     int head_split;         // blocks per tile along the heads (>= 1); set by the launcher
     int order;              // block order; set by the launcher
 };
@@ -57,6 +71,7 @@ struct MetricParams {
     int chunk_vecs;
     int n_units;
     SelectParams sel;
+    int pdl;                      // PDL_TRIGGER: dependents may start once every block streams
 };
 
 // Phase 2 of the two-phase exchange: up to three tensors, src = [2][S][H][D] (the

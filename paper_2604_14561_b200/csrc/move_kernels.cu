@@ -69,6 +69,15 @@ __device__ __forceinline__ void st_row(uint4 *p, const uint4 v) {
     if (HINT == 2) *p = v; else __stcs(p, v);
 }
 
+// Runs griddepcontrol.wait when the thread leaves the kernel (any return path).
+struct PdlTail {
+    int flags;
+    __device__ __forceinline__ explicit PdlTail(int f) : flags(f) {}
+    __device__ __forceinline__ ~PdlTail() {
+        if (flags & PDL_WAIT_AT_END) asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
+};
+
 template <int U>
 struct UnrollTag { static constexpr int value = U; };
 
@@ -85,11 +94,17 @@ __global__ void __launch_bounds__(THREADS, MINB) move_rows_kernel(const __grid_c
     constexpr int D = LPR * 8;
     constexpr int TOK = THREADS / LPR;  // token slots per tile
 
+    if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
+    PdlTail tail(p.pdl);  // PDL_WAIT_AT_END: every exit path waits for the predecessor first
+
     int n_valid = p.n_slots;
     long long src_head = p.src_head, dst_head = p.dst_head;
     if (p.map != MAP_FULL) {
-        const long long nv = (long long)__ldg(p.n_active) * p.T;
+        // written by the preceding kernel: an ordinary (coherent) load, ordered after griddepcontrol.wait
+        const long long nv = (long long)__ldcg(p.n_active) * p.T;
         n_valid = nv < (long long)p.n_slots ? (int)nv : p.n_slots;
+        if (n_valid < 0) n_valid = 0;
         if (src_head == COMPACT_STRIDE) src_head = (long long)n_valid * D;
         if (dst_head == COMPACT_STRIDE) dst_head = (long long)n_valid * D;
     }
@@ -126,7 +141,9 @@ __global__ void __launch_bounds__(THREADS, MINB) move_rows_kernel(const __grid_c
     long long s = o, d = o;
     if (p.map != MAP_FULL) {
         const int a = o / p.T;
-        const long long tk = (long long)__ldg(p.idx + a) * p.T + (o - a * p.T);
+        int unit = __ldcg(p.idx + a);  // a list that was never written must not send accesses out of bounds
+        unit = unit < 0 ? 0 : (unit >= p.n_units ? p.n_units - 1 : unit);
+        const long long tk = (long long)unit * p.T + (o - a * p.T);
         if (p.map == MAP_GATHER) s = tk; else d = tk;
     }
     const uint4 *sp = reinterpret_cast<const uint4 *>(job.src + s * p.src_tok) + lr + h_lo * sh;
@@ -226,6 +243,18 @@ cudaError_t launch_variant(MoveParams p, cudaStream_t stream, int head_split = 1
     const long long blocks = tiles * head_split * p.njobs;
     if (blocks == 0) return cudaSuccess;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    if (p.pdl & PDL_LAUNCH_ATTR) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)blocks);
+        cfg.blockDim = dim3(THREADS);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, move_rows_kernel<LPR, KIND, UN, UP, THREADS, MINB, HINT>, p);
+    }
     move_rows_kernel<LPR, KIND, UN, UP, THREADS, MINB, HINT><<<(unsigned)blocks, THREADS, 0, stream>>>(p);
     return cudaGetLastError();
 }

@@ -257,6 +257,10 @@ vmajor_metric_kernel(const __grid_constant__ MetricParams p, const int fuse_sele
         if (lane == 0 && acc != 0) atomicAdd(p.acc + u, acc);
     }
 
+    // This block has streamed its share: a dependent launch may begin to occupy
+    // the SMs (it orders itself behind the whole grid with griddepcontrol.wait).
+    if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     // The block that draws the last ticket sees every accumulator complete.
     __threadfence();
     __syncthreads();
