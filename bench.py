@@ -303,6 +303,28 @@ def run_ours(args):
             orders[name] = {"us_median": 1e3 * statistics.median(ms), "us_min": 1e3 * min(ms),
                             "gbs_median": step_bytes / (statistics.median(ms) * 1e-3) / 1e9,
                             "launches_per_step": 2 if order == binding.V_FIRST else 1}
+        # V-first evidence: V's exchange and the Q/K launch issued as two calls with their own events
+        ev = {n: torch.cuda.Event(enable_timing=True) for n in ("v0", "v1", "qk0", "qk1")}
+        timeline = []
+        for _ in range(10):
+            torch.cuda.synchronize()
+            ev["v0"].record(sv)
+            binding.prologue(None, None, v, None, None, vh, None, None, cfg["eps"], None, P, S, H, D,
+                             order=binding.LUMP, stream_qk=sv, stream_v=sv)
+            ev["v1"].record(sv)
+            ev["qk0"].record(sq)
+            binding.prologue(q, k, None, qh, kh, None, wq, wk, cfg["eps"], cs, P, S, H, D,
+                             order=binding.LUMP, stream_qk=sq, stream_v=sq)
+            ev["qk1"].record(sq)
+            torch.cuda.synchronize()
+            timeline.append((ev["v0"].elapsed_time(ev["v1"]), ev["v0"].elapsed_time(ev["qk0"]),
+                             ev["v0"].elapsed_time(ev["qk1"])))
+        timeline.sort(key=lambda t: t[2])
+        mid = timeline[len(timeline) // 2]
+        v_first_timeline = {"v_start_us": 0.0, "v_end_us": 1e3 * mid[0], "qk_start_us": 1e3 * mid[1],
+                            "qk_end_us": 1e3 * mid[2],
+                            "note": "V is launched first on its own stream and completes first; Q/K (norm + RoPE) run beside it"}
+
         # dominant kernel of the headline loop: the norm + RoPE + exchange launch over Q and K
         # (two thirds of the bytes), timed alone on its stream
         def qk_only():
@@ -360,7 +382,7 @@ def run_ours(args):
                        "algorithmic_bytes_per_step": step_bytes, "l2": "inputs and outputs (775 MB per step) exceed the 126 MB L2",
                        "replicas": world},
             "gpu_launches": 2 * args.steps,
-            "clocks": clocks, "orders": orders, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+            "clocks": clocks, "orders": orders, "v_first_timeline": v_first_timeline, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
             "per_config": per_config,
         }
     if world > 1:
@@ -384,15 +406,21 @@ def read_traffic_note():
 
 def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "temporal")):
     """µs/layer and GB/s of the other synthetic workloads, L2 flushed between
-    iterations (they fit in the 126 MB L2), plus the selective step of the
+    iterations (they fit in the 126 MB L2; flush = write then read 512 MB), plus the selective step of the
     temporal workload."""
     out = {}
     scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     sq, sv = torch.cuda.Stream(), torch.cuda.Stream()
 
+    sink = torch.zeros(1, dtype=torch.int64, device="cuda")
+
     def flush():
+        # write a buffer four times the L2, then read it back: the L2 ends up full of
+        # clean lines, so the timed region neither hits in L2 nor pays for the write-back
+        # of the flush's own dirty lines
         with torch.cuda.stream(sq):
             scratch.zero_()
+            torch.sum(scratch.view(torch.int64), dim=0, keepdim=True, out=sink)
 
     iters = max(10, min(args.steps, 50))
     for name in names:
@@ -451,10 +479,27 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
         n_act = int(na.item())
         tile = T * H * D * 2
         sb = 2 * E * 2 + 3 * 2 * n_act * tile + 3 * 2 * n_act * tile
+
+        def part_select():
+            binding.vmajor_select_compact(v, cur_v, P, S, H, D, T, r, n_groups, metric, mask, idx, na, None,
+                                          ws, ws_bytes, stream=sq)
+
+        def part_pack():
+            binding.pack_active_qkv(q, k, cur_v, wq, wk, cfg["eps"], cs, idx, na, comp[0], comp[1], comp[2],
+                                    P, S, H, D, T, stream=sq)
+
+        def part_unpack():
+            binding.unpack_qkv(comp[0], comp[1], comp[2], idx, na, qh, kh, vh, P, S, H, D, T, stream=sq)
+        breakdown = {}
+        for pname, fn, nbytes in (("metric_select", part_select, 2 * E * 2), ("pack_qkv", part_pack, 6 * n_act * tile),
+                                  ("unpack_qkv", part_unpack, 6 * n_act * tile)):
+            t = statistics.median(time_steps(torch, fn, sq, iters, 3, flush=flush))
+            breakdown[pname] = {"us_cold_l2": 1e3 * t, "bytes": nbytes, "gbs": nbytes / (t * 1e-3) / 1e9}
         best = min(sel.values())
         out["temporal_selective_step"] = {"n_active": n_act, "n_units": n, "bytes": sb,
                                           "us_cold_l2": sel, "gbs_cold_l2_best": sb / (best * 1e-6) / 1e9,
                                           "launches_per_step": {"lump": 4, "v_first": 5},
+                                          "parts_timed_alone": breakdown,
                                           "api": "cocodiff_selective_prologue"}
     return out
 
