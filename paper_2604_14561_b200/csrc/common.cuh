@@ -87,7 +87,9 @@ struct TapaParams {
 cudaError_t launch_tapa_phase2(const TapaParams &p, int D, cudaStream_t stream);
 cudaError_t launch_move(const MoveParams &p, int D, cudaStream_t stream);
 cudaError_t launch_rope_table(float *cs, const int32_t *pos, int S, int D, double theta, cudaStream_t stream);
-cudaError_t launch_select(const SelectParams &p, cudaStream_t stream);
+// pdl: PDL_LAUNCH_ATTR | PDL_WAIT_AT_START when the metric was produced by the preceding
+// kernel of the stream; PDL_TRIGGER lets the kernel after the selection start early.
+cudaError_t launch_select(const SelectParams &p, cudaStream_t stream, int pdl = 0);
 cudaError_t launch_metric_select(const MetricParams &p, cudaStream_t stream);
 
 }  // namespace cocodiff

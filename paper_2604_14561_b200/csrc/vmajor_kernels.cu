@@ -193,15 +193,19 @@ __device__ void select_group_large(const SelectParams &p, int grp, SelectSmem &s
     emit_selection<BLOCK>(p, grp, vals, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm.warp_sums);
 }
 
-__global__ void __launch_bounds__(256) vmajor_select_small_kernel(const __grid_constant__ SelectParams p) {
+__global__ void __launch_bounds__(256) vmajor_select_small_kernel(const __grid_constant__ SelectParams p, const int pdl) {
     __shared__ SelectSmem sm;
+    if (pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
     select_group_small<256>(p, blockIdx.x, sm);
 }
 
 constexpr int kLargeBlock = 1024;
 __global__ void __launch_bounds__(kLargeBlock)
-vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int staged) {
+vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int staged, const int pdl) {
     __shared__ SelectSmem sm;
+    if (pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
     __shared__ int warp_hist[(kLargeBlock / 32) * 256];
     extern __shared__ unsigned long long dyn_vals[];
     select_group_large<kLargeBlock>(p, blockIdx.x, sm, dyn_vals, warp_hist, staged);
@@ -279,12 +283,28 @@ vmajor_metric_kernel(const __grid_constant__ MetricParams p, const int fuse_sele
 
 }  // namespace
 
-cudaError_t launch_select(const SelectParams &p, cudaStream_t stream) {
+namespace {
+template <typename... Args>
+cudaError_t launch_maybe_programmatic(void (*kernel)(Args...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                      int pdl, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (pdl & PDL_LAUNCH_ATTR) ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+}  // namespace
+
+cudaError_t launch_select(const SelectParams &p, cudaStream_t stream, int pdl) {
     if (p.n == 0) return cudaMemsetAsync(p.n_active, 0, sizeof(int32_t), stream);
-    if (p.g <= kCountMax) {
-        vmajor_select_small_kernel<<<p.n_groups, 256, 0, stream>>>(p);
-        return cudaGetLastError();
-    }
+    if (p.g <= kCountMax)
+        return launch_maybe_programmatic(vmajor_select_small_kernel, dim3(p.n_groups), dim3(256), 0, stream, pdl, p, pdl);
     // stage the group's metrics in shared memory when they fit beside the histograms
     const size_t want = (size_t)p.g * sizeof(unsigned long long);
     const size_t limit = 160 * 1024;
@@ -299,8 +319,8 @@ cudaError_t launch_select(const SelectParams &p, cudaStream_t stream) {
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    vmajor_select_large_kernel<<<p.n_groups, kLargeBlock, dyn, stream>>>(p, staged);
-    return cudaGetLastError();
+    return launch_maybe_programmatic(vmajor_select_large_kernel, dim3(p.n_groups), dim3(kLargeBlock), dyn, stream, pdl,
+                                     p, staged, pdl);
 }
 
 cudaError_t launch_metric_select(const MetricParams &p, cudaStream_t stream) {
@@ -319,7 +339,8 @@ cudaError_t launch_metric_select(const MetricParams &p, cudaStream_t stream) {
     vmajor_metric_kernel<<<(unsigned)blocks, kMetricThreads, 0, stream>>>(p, fuse);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || fuse) return e;
-    return launch_select(p.sel, stream);
+    // the separate selection kernel consumes the metric of the kernel just launched
+    return launch_select(p.sel, stream, PDL_LAUNCH_ATTR | PDL_WAIT_AT_START | (p.pdl & PDL_TRIGGER));
 }
 
 }  // namespace cocodiff
