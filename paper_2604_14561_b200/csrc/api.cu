@@ -138,6 +138,12 @@ size_t vmajor_ws_bytes(int S, int T) {
     return ((n * 8 + 255) / 256) * 256 + 256;  // accumulators, then the ticket
 }
 
+// Token slots that the selection rule leaves active: (n - n_groups * floor(r * g)) * T.
+int active_slots(int S, int T, double r, int n_groups) {
+    const int n = S / T, g = n / n_groups;
+    return (n - n_groups * (int)std::floor(r * (double)g)) * T;
+}
+
 int check_select(const uint16_t *prev_v, const uint16_t *cur_v, int P, int S, int H, int D, int T, double r,
                  int n_groups, const uint64_t *metric, const uint8_t *mask, const int32_t *idx,
                  const int32_t *n_active, const void *workspace, size_t workspace_bytes) {
@@ -471,9 +477,9 @@ int cocodiff_vmajor_select_compact(const uint16_t *prev_v, const uint16_t *cur_v
     rc = enqueue_metric_select(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, st,
                                v_compact ? PDL_TRIGGER : 0);
     if (rc) return rc;
-    if (v_compact)
-        return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, S, S, H, D, T, st,
-                            PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
+    if (v_compact)  // the host knows how many units the rule leaves active: exact grid
+        return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, active_slots(S, T, r, n_groups), S,
+                            H, D, T, st, PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
     return COCODIFF_OK;
 }
 
@@ -573,8 +579,7 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
                     return COCODIFF_ALIASING;
     }
     // the host knows how many units will be active: grids are sized exactly
-    const int n = S / T, g = n / n_groups;
-    const int slots = (n - n_groups * (int)std::floor(r * (double)g)) * T;
+    const int slots = active_slots(S, T, r, n_groups);
     cudaStream_t sq = (cudaStream_t)stream_qk, sv = (cudaStream_t)stream_v;
     // On one stream the three kernels are chained with programmatic dependent launches:
     // each successor becomes resident while its predecessor drains and orders itself
@@ -773,9 +778,9 @@ int cocodiff_vmajor_select_compact_static(const uint16_t *prev_v, const uint16_t
     rc = enqueue_metric_select(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, scratch, st,
                                v_compact ? PDL_TRIGGER : 0);
     if (rc) return rc;
-    if (v_compact)
-        return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, S, S, H, D, T, st,
-                            PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
+    if (v_compact)  // the host knows how many units the rule leaves active: exact grid
+        return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, active_slots(S, T, r, n_groups), S,
+                            H, D, T, st, PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
     return COCODIFF_OK;
 }
 
