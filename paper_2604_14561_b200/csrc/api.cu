@@ -172,9 +172,9 @@ int check_tiles(const uint16_t *const in[3], uint16_t *const out[3], int S, int 
     return check_pairs(in, out, (size_t)S * H * D * 2);
 }
 
-int enqueue_metric_select(const uint16_t *prev_v, const uint16_t *cur_v, int S, int H, int D, int T, double r,
-                          int n_groups, uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
-                          void *workspace, cudaStream_t st, int pdl = 0) {
+MetricParams make_metric_params(const uint16_t *prev_v, const uint16_t *cur_v, int S, int H, int D, int T, double r,
+                                int n_groups, uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
+                                void *workspace) {
     const int n = S / T;
     const size_t need = vmajor_ws_bytes(S, T);
     MetricParams mp;
@@ -196,17 +196,23 @@ int enqueue_metric_select(const uint16_t *prev_v, const uint16_t *cur_v, int S, 
     mp.sel.mask = mask;
     mp.sel.idx = idx;
     mp.sel.n_active = n_active;
+    return mp;
+}
+
+int enqueue_metric_select(const uint16_t *prev_v, const uint16_t *cur_v, int S, int H, int D, int T, double r,
+                          int n_groups, uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
+                          void *workspace, cudaStream_t st, int pdl = 0) {
+    MetricParams mp = make_metric_params(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace);
     mp.pdl = pdl;
-    CK(cudaMemsetAsync(workspace, 0, need, st));
+    CK(cudaMemsetAsync(workspace, 0, vmajor_ws_bytes(S, T), st));
     CK(launch_metric_select(mp, st));
     return COCODIFF_OK;
 }
 
 // Compaction of up to three tensors in one launch; slot order (Q, K, V), V's blocks first.
-int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint16_t *wq, const uint16_t *wk,
-                 float eps, const float *cs, const int32_t *idx, const int32_t *n_active, int slots, int S,
-                 int H, int D, int T, cudaStream_t st, int pdl = 0) {
-    (void)S;
+MoveParams make_pack_params(const uint16_t *const in[3], uint16_t *const out[3], const uint16_t *wq,
+                            const uint16_t *wk, float eps, const float *cs, const int32_t *idx,
+                            const int32_t *n_active, int slots, int S, int H, int D, int T) {
     MoveParams p;
     std::memset(&p, 0, sizeof p);
     p.n_slots = slots;
@@ -218,7 +224,6 @@ int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint
     p.map = MAP_GATHER;
     p.T = T;
     p.n_units = S / T;
-    p.pdl = pdl;
     p.idx = idx;
     p.n_active = n_active;
     p.cs = cs;
@@ -226,13 +231,21 @@ int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint
     if (in[2]) p.job[p.njobs++] = MoveJob{in[2], out[2], nullptr};
     if (in[0]) p.job[p.njobs++] = MoveJob{in[0], out[0], wq};
     if (in[1]) p.job[p.njobs++] = MoveJob{in[1], out[1], wk};
+    return p;
+}
+
+int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint16_t *wq, const uint16_t *wk,
+                 float eps, const float *cs, const int32_t *idx, const int32_t *n_active, int slots, int S,
+                 int H, int D, int T, cudaStream_t st, int pdl = 0) {
+    MoveParams p = make_pack_params(in, out, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T);
+    p.pdl = pdl;
     if (p.njobs == 0) return COCODIFF_OK;
     CK(launch_move(p, D, st));
     return COCODIFF_OK;
 }
 
-int enqueue_unpack(const uint16_t *const in[3], uint16_t *const out[3], const int32_t *idx,
-                   const int32_t *n_active, int slots, int S, int H, int D, int T, cudaStream_t st, int pdl = 0) {
+MoveParams make_unpack_params(const uint16_t *const in[3], uint16_t *const out[3], const int32_t *idx,
+                              const int32_t *n_active, int slots, int S, int H, int D, int T) {
     MoveParams p;
     std::memset(&p, 0, sizeof p);
     p.n_slots = slots;
@@ -244,11 +257,17 @@ int enqueue_unpack(const uint16_t *const in[3], uint16_t *const out[3], const in
     p.map = MAP_SCATTER;
     p.T = T;
     p.n_units = S / T;
-    p.pdl = pdl;
     p.idx = idx;
     p.n_active = n_active;
     for (int i = 2; i >= 0; --i)
         if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr};
+    return p;
+}
+
+int enqueue_unpack(const uint16_t *const in[3], uint16_t *const out[3], const int32_t *idx,
+                   const int32_t *n_active, int slots, int S, int H, int D, int T, cudaStream_t st, int pdl = 0) {
+    MoveParams p = make_unpack_params(in, out, idx, n_active, slots, S, H, D, T);
+    p.pdl = pdl;
     if (p.njobs == 0) return COCODIFF_OK;
     CK(launch_move(p, D, st));
     return COCODIFF_OK;

@@ -1,0 +1,212 @@
+// Device code of the row mover (see move_kernels.cu for the description of the
+// kernel built from it): the per-block work, separate from the launch code.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace cocodiff {
+namespace rows {
+
+// eight bf16 values of a 16-byte vector, widened exactly
+__device__ __forceinline__ void unpack8(const uint4 v, float (&x)[8]) {
+    x[0] = __uint_as_float(v.x << 16);
+    x[1] = __uint_as_float(v.x & 0xffff0000u);
+    x[2] = __uint_as_float(v.y << 16);
+    x[3] = __uint_as_float(v.y & 0xffff0000u);
+    x[4] = __uint_as_float(v.z << 16);
+    x[5] = __uint_as_float(v.z & 0xffff0000u);
+    x[6] = __uint_as_float(v.w << 16);
+    x[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+
+// two floats -> packed bf16x2, round to nearest even, lo in the low half
+__device__ __forceinline__ unsigned pack2(float lo, float hi) {
+    const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const unsigned *>(&b);
+}
+
+// 1/sqrt(x) for x > 0 (x = mean square + eps): one MUFU, relative error < 2^-22
+__device__ __forceinline__ float rsqrt_approx(float x) {
+    float y;
+    asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Sum over the LPR lanes that hold one row; the whole warp takes part.
+template <int LPR>
+__device__ __forceinline__ float group_sum(float v) {
+#pragma unroll
+    for (int off = LPR / 2; off >= 1; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    return v;
+}
+
+// What a launch may contain: plain moves only, norm + RoPE jobs only, or both
+// (the lump order of issue).  The specialised forms need fewer registers.
+enum JobKind : int { KIND_PLAIN = 0, KIND_NORM = 1, KIND_MIXED = 2 };
+
+// HINT selects the cache policy of the streaming accesses (0: evict-first loads
+// and stores, 1: read-only path loads + evict-first stores, 2: default, 3: loads
+// served by the L2 only).  The policies measured the same on B200; 0 is used.
+template <int HINT>
+__device__ __forceinline__ uint4 ld_row(const uint4 *p) {
+    if (HINT == 0) return __ldcs(p);
+    if (HINT == 1) return __ldg(p);
+    if (HINT == 3) return __ldcg(p);  // L2 only: data written earlier in the same launch by other blocks
+    return *p;
+}
+template <int HINT>
+__device__ __forceinline__ void st_row(uint4 *p, const uint4 v) {
+    if (HINT == 2) *p = v; else __stcs(p, v);
+}
+
+template <int U>
+struct UnrollTag { static constexpr int value = U; };
+
+// Walks heads [h, h_hi) in groups of U (all loads of a group are issued before
+// its stores), then halves U for what is left, down to single heads.
+template <int U, typename F>
+__device__ __forceinline__ void heads_loop(int &h, const int h_hi, F &&body) {
+    for (; h + U <= h_hi; h += U) body(UnrollTag<U>{});
+    if constexpr (U > 1) heads_loop<U / 2>(h, h_hi, body);
+}
+
+// One block's share of a move: block id b -> (job, head range, token tile).
+// LPR lanes per row (D = 8 * LPR); KIND: what the launch contains; UN / UP = heads
+// in flight per thread on the norm path / the plain path.  TOK = THREADS / LPR
+// token slots per tile.  Callable from any kernel whose blocks have THREADS threads.
+template <int LPR, int KIND, int UN, int UP, int THREADS, int HINT>
+__device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b) {
+    constexpr int D = LPR * 8;
+    constexpr int TOK = THREADS / LPR;  // token slots per tile
+
+    int n_valid = p.n_slots;
+    long long src_head = p.src_head, dst_head = p.dst_head;
+    if (p.map != MAP_FULL) {
+        // written by the preceding kernel: an ordinary (coherent) load, ordered after griddepcontrol.wait
+        const long long nv = (long long)__ldcg(p.n_active) * p.T;
+        n_valid = nv < (long long)p.n_slots ? (int)nv : p.n_slots;
+        if (n_valid < 0) n_valid = 0;
+        if (src_head == COMPACT_STRIDE) src_head = (long long)n_valid * D;
+        if (dst_head == COMPACT_STRIDE) dst_head = (long long)n_valid * D;
+    }
+    // Block id -> (job, head range, token tile).  ORDER 0: job-major (all of V,
+    // then Q, then K); 1: head-range-major (V, Q, K tiles of range 0, then range 1 ...);
+    // 2: tile-major (the jobs and ranges of one tile are neighbours).
+    const unsigned tiles = (unsigned)(p.n_slots + TOK - 1) / TOK;
+    const unsigned hsplit = (unsigned)p.head_split, njobs = (unsigned)p.njobs;
+    unsigned tile, y, job_i;
+    {
+        if (p.order == 0) { job_i = b / (tiles * hsplit); const unsigned r = b - job_i * tiles * hsplit; y = r / tiles; tile = r - y * tiles; }
+        else if (p.order == 1) { y = b / (tiles * njobs); const unsigned r = b - y * tiles * njobs; job_i = r / tiles; tile = r - job_i * tiles; }
+        else { tile = b / (njobs * hsplit); const unsigned r = b - tile * njobs * hsplit; job_i = r / hsplit; y = r - job_i * hsplit; }
+    }
+    const int tile0 = (int)tile * TOK;
+    if (tile0 >= n_valid) return;  // block-uniform: nothing in this tile
+    const long long sh = src_head / 8, dh = dst_head / 8;  // head strides in vectors
+    const int lr = (int)threadIdx.x % LPR;
+
+    // heads [h_lo, h_hi) of this block
+    const int hs = (p.H + (int)hsplit - 1) / (int)hsplit;
+    const int h_lo = (int)y * hs;
+    const int h_hi = h_lo + hs < p.H ? h_lo + hs : p.H;
+    const MoveJob job = job_i == 0 ? p.job[0] : (job_i == 1 ? p.job[1] : p.job[2]);
+
+    // A slot past the end keeps its lanes in step with the warp (the row
+    // reduction uses full-warp shuffles): it re-reads the tile's first slot
+    // and stores nothing.
+    const int o_raw = tile0 + (int)threadIdx.x / LPR;
+    const bool valid = o_raw < n_valid;
+    const int o = valid ? o_raw : tile0;
+
+    long long s = o, d = o;
+    if (p.map != MAP_FULL) {
+        const int a = o / p.T;
+        int unit = __ldcg(p.idx + a);  // a list that was never written must not send accesses out of bounds
+        unit = unit < 0 ? 0 : (unit >= p.n_units ? p.n_units - 1 : unit);
+        const long long tk = (long long)unit * p.T + (o - a * p.T);
+        if (p.map == MAP_GATHER) s = tk; else d = tk;
+    }
+    const uint4 *sp = reinterpret_cast<const uint4 *>(job.src + s * p.src_tok) + lr + h_lo * sh;
+    uint4 *dp = reinterpret_cast<uint4 *>(job.dst + d * p.dst_tok) + lr + h_lo * dh;
+
+    if (KIND == KIND_PLAIN || (KIND == KIND_MIXED && job.w == nullptr)) {
+        if (!valid) return;
+        int h = h_lo;
+        heads_loop<UP>(h, h_hi, [&](auto u_tag) {
+            constexpr int U = decltype(u_tag)::value;
+            uint4 v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) { v[u] = ld_row<HINT>(sp); sp += sh; }
+#pragma unroll
+            for (int u = 0; u < U; ++u) { st_row<HINT>(dp, v[u]); dp += dh; }
+        });
+        return;
+    }
+
+    // Per-token constants, reused for all heads: the norm weight folded into the
+    // rotation.  With pair q = elements (2q, 2q+1) = (a_q, b_q):
+    //   out[2q] = inv * (a_q*ka_q + b_q*kb_q),  out[2q+1] = inv * (a_q*kc_q + b_q*kd_q).
+    // Pairs (0,1) and (2,3) are processed together with sm_100's packed fp32x2
+    // arithmetic (two independent IEEE fp32 operations per instruction).
+    float2 ka01, kb01, kc01, kd01, ka23, kb23, kc23, kd23;
+    {
+        float w[8];
+        unpack8(__ldg(reinterpret_cast<const uint4 *>(job.w) + lr), w);
+        float c[4] = {1.f, 1.f, 1.f, 1.f}, sn[4] = {0.f, 0.f, 0.f, 0.f};
+        if (p.cs != nullptr) {
+            // pairs 4*lr .. 4*lr+3 of token s: 8 floats (cos, sin, cos, sin, ...)
+            const float4 *tb = reinterpret_cast<const float4 *>(p.cs + s * D) + 2 * lr;
+            const float4 t0 = __ldg(tb), t1 = __ldg(tb + 1);
+            c[0] = t0.x; sn[0] = t0.y; c[1] = t0.z; sn[1] = t0.w;
+            c[2] = t1.x; sn[2] = t1.y; c[3] = t1.z; sn[3] = t1.w;
+        }
+        ka01 = make_float2(w[0] * c[0], w[2] * c[1]);
+        kb01 = make_float2(-(w[1] * sn[0]), -(w[3] * sn[1]));
+        kc01 = make_float2(w[0] * sn[0], w[2] * sn[1]);
+        kd01 = make_float2(w[1] * c[0], w[3] * c[1]);
+        ka23 = make_float2(w[4] * c[2], w[6] * c[3]);
+        kb23 = make_float2(-(w[5] * sn[2]), -(w[7] * sn[3]));
+        kc23 = make_float2(w[4] * sn[2], w[6] * sn[3]);
+        kd23 = make_float2(w[5] * c[2], w[7] * c[3]);
+    }
+    const float inv_d = 1.0f / (float)D;
+    const float eps = p.eps;
+
+    auto norm_rope_row = [&](const uint4 v) -> uint4 {
+        // a_q = low bf16 of word q, b_q = high bf16 of word q, widened exactly
+        const float2 a01 = make_float2(__uint_as_float(v.x << 16), __uint_as_float(v.y << 16));
+        const float2 b01 = make_float2(__uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y & 0xffff0000u));
+        const float2 a23 = make_float2(__uint_as_float(v.z << 16), __uint_as_float(v.w << 16));
+        const float2 b23 = make_float2(__uint_as_float(v.z & 0xffff0000u), __uint_as_float(v.w & 0xffff0000u));
+        float2 acc = __fmul2_rn(a01, a01);
+        acc = __ffma2_rn(b01, b01, acc);
+        acc = __ffma2_rn(a23, a23, acc);
+        acc = __ffma2_rn(b23, b23, acc);
+        const float ss = group_sum<LPR>(acc.x + acc.y);
+        const float inv = rsqrt_approx(fmaf(ss, inv_d, eps));
+        const float2 inv2 = make_float2(inv, inv);
+        const float2 lo01 = __fmul2_rn(__ffma2_rn(a01, ka01, __fmul2_rn(b01, kb01)), inv2);
+        const float2 hi01 = __fmul2_rn(__ffma2_rn(a01, kc01, __fmul2_rn(b01, kd01)), inv2);
+        const float2 lo23 = __fmul2_rn(__ffma2_rn(a23, ka23, __fmul2_rn(b23, kb23)), inv2);
+        const float2 hi23 = __fmul2_rn(__ffma2_rn(a23, kc23, __fmul2_rn(b23, kd23)), inv2);
+        return make_uint4(pack2(lo01.x, hi01.x), pack2(lo01.y, hi01.y), pack2(lo23.x, hi23.x), pack2(lo23.y, hi23.y));
+    };
+
+    int h = h_lo;
+    heads_loop<UN>(h, h_hi, [&](auto u_tag) {
+        constexpr int U = decltype(u_tag)::value;
+        uint4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) { v[u] = ld_row<HINT>(sp); sp += sh; }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const uint4 y = norm_rope_row(v[u]);
+            if (valid) st_row<HINT>(dp, y);
+            dp += dh;
+        }
+    });
+}
+
+}  // namespace rows
+}  // namespace cocodiff
