@@ -7,7 +7,14 @@ namespace cocodiff {
 namespace vmajor {
 
 constexpr int kMetricThreads = 256;
-constexpr int kMetricUnroll = 4;
+#ifndef COCODIFF_METRIC_UNROLL
+#define COCODIFF_METRIC_UNROLL 4
+#endif
+#ifndef COCODIFF_METRIC_BLOCKS_PER_SM
+#define COCODIFF_METRIC_BLOCKS_PER_SM 4
+#endif
+constexpr int kMetricUnroll = COCODIFF_METRIC_UNROLL;
+constexpr int kMetricBlocksPerSm = COCODIFF_METRIC_BLOCKS_PER_SM;
 constexpr int kCountMax = 512;  // groups up to this size are ranked by counting
 
 struct SelectSmem {

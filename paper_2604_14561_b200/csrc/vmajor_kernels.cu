@@ -35,7 +35,7 @@ vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int sta
     select_group_large<kLargeBlock>(p, blockIdx.x, sm, dyn_vals, warp_hist, staged);
 }
 
-__global__ void __launch_bounds__(kMetricThreads, 4)
+__global__ void __launch_bounds__(kMetricThreads, kMetricBlocksPerSm)
 vmajor_metric_kernel(const __grid_constant__ MetricParams p, const int fuse_select) {
     __shared__ SelectSmem sm;
     __shared__ int is_last;
@@ -111,7 +111,7 @@ cudaError_t launch_metric_select(const MetricParams &p, cudaStream_t stream) {
     long long blocks = (total + (kMetricThreads / 32) - 1) / (kMetricThreads / 32);
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const long long cap = (long long)sms * 4;
+    const long long cap = (long long)sms * kMetricBlocksPerSm;
     if (blocks > cap) blocks = cap;
     // one small group: its selection rides in the metric kernel's last block; several
     // groups or a large one go to their own launch, one block per group
