@@ -240,6 +240,11 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        from paper_2604_14561_b200 import build as cuda_build
+        cuda_build.build()            # no-op when libcocodiff.so is newer than its sources
+    if world > 1:
+        dist.barrier()
     binding.lib()
 
     cfg = synth.config(WORKLOAD)
