@@ -70,6 +70,8 @@ int cocodiff_rope_table_2d(float *cs, const int32_t *pos, int S, int D, double t
 /* QK normalisation + RoPE alone (Section II-B), SEQ in -> SEQ out.
  * y = RoPE(x * rsqrt(mean_D(x^2) + eps) * w), per (token, head), fp32 arithmetic,
  * one round-to-nearest-even to bf16.  Pair (2p, 2p+1) is rotated by cs[s][p].
+ * Inputs are expected finite with squares representable in fp32 (|x| < 1.8e19);
+ * NaN, Inf and eps = 0 with an all-zero row give unspecified bit patterns.
  * q/k may be NULL to skip that tensor; out == in (same tensor) is allowed,
  * any other overlap is COCODIFF_ALIASING.  wq, wk: [D] bf16.  cs may be NULL
  * (no rotation). */
