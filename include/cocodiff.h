@@ -280,6 +280,24 @@ int cocodiff_vmajor_select_compact_static(const uint16_t *prev_v, const uint16_t
                                           uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
                                           uint16_t *v_compact, void *stream);
 
+/* Diagnostic for the bounds-checked build of this library (compiled with
+ * -DCOCODIFF_DEBUG_BOUNDS; build.py --debug-bounds writes libcocodiff_debug.so).
+ * (The paper has no counterpart.)  In that build every global access of every
+ * kernel is checked against the extent of the buffer it belongs to; an access
+ * outside is counted and skipped, never performed and never trapped.  This
+ * call waits for the device, returns the number of such accesses on the current
+ * device since the previous call and resets the counter; -2 on a CUDA error.
+ * The normal build carries no checks: there the call returns -1. */
+long long cocodiff_debug_bounds_violations(void);
+
+/* Self-test of that checker (bounds-checked build only; -1 in the normal build,
+ * -2 on bad arguments or a CUDA error): moves x [S][H][D] to y while claiming
+ * that both buffers end after S/2 tokens.  The accesses beyond are in fact
+ * inside the caller's buffers, so nothing is harmed; the checker must count
+ * and skip each of them.  Returns the count: 2 * (S - S/2) * H * D/8 (one load
+ * and one store per 16-byte vector); y keeps its old contents beyond S/2. */
+long long cocodiff_debug_bounds_selftest(const uint16_t *x, uint16_t *y, int S, int H, int D, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

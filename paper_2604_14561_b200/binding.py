@@ -46,6 +46,8 @@ SIGNATURES = {
     "cocodiff_layer_step": (_I, [_I] * 4 + [_P] * 6 + [_F, _P] + [_I] * 6 + [_P] * 11 + [_Z, _I, _P, _P, _P]),
     "cocodiff_tapa_phase1": (_I, [_P] * 6 + [_I] * 4 + [_P]),
     "cocodiff_tapa_phase2": (_I, [_P] * 6 + [_I] * 4 + [_P]),
+    "cocodiff_debug_bounds_violations": (C.c_longlong, []),
+    "cocodiff_debug_bounds_selftest": (C.c_longlong, [_P, _P, _I, _I, _I, _P]),
     "cocodiff_selective_prologue": (_I, [_P] * 6 + [_F, _P] + [_I] * 5 + [_D, _I] + [_P] * 11 + [_Z, _I, _P, _P]),
 }
 
@@ -236,3 +238,15 @@ def layer_step(step, total_steps, warmup, sync_interval, prev_v, q, k, v, wq, wk
                _ptr(k_cache), _ptr(v_cache), _ptr(workspace), workspace_bytes, order, _stream(stream_qk),
                _stream(stream_v), C.cast(C.byref(sent), C.c_void_p), check=check)
     return rc, int(sent.value)
+
+
+def debug_bounds_violations() -> int:
+    """Out-of-bounds accesses caught (and skipped) by the bounds-checked build since the
+    last call; -1 when the loaded library is the normal build."""
+    return int(lib().cocodiff_debug_bounds_violations())
+
+
+def debug_bounds_selftest(x, y, S, H, D, stream=None) -> int:
+    """Bounds-checked build only: a move told that its buffers end after S/2 tokens;
+    returns how many accesses the checker caught and skipped (-1 in the normal build)."""
+    return int(lib().cocodiff_debug_bounds_selftest(_ptr(x), _ptr(y), S, H, D, _stream(stream)))

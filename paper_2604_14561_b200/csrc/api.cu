@@ -69,6 +69,34 @@ int get_events(ForkJoin **out) {
     return COCODIFF_OK;
 }
 
+// Bounds-checked build: one violation counter per device, inside the library image.
+#ifdef COCODIFF_DEBUG_BOUNDS
+static __device__ unsigned long long g_bounds_violations;
+unsigned long long *debug_counter() {
+    static std::mutex mu;
+    static unsigned long long *addr[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_bounds_violations) != cudaSuccess) return nullptr;
+        addr[dev] = static_cast<unsigned long long *>(ptr);
+    }
+    return addr[dev];
+}
+#else
+unsigned long long *debug_counter() { return nullptr; }
+#endif
+
+// Extents (in elements / floats) of the buffers a move touches, for the bounds-checked build.
+void set_extents(MoveParams &p, long long src, long long dst, long long cs) {
+    p.src_extent = src;
+    p.dst_extent = dst;
+    p.cs_extent = cs;
+    p.debug = debug_counter();
+}
+
 MoveParams seq_to_head(int S, int H, int D) {
     MoveParams p;
     std::memset(&p, 0, sizeof p);
@@ -80,6 +108,7 @@ MoveParams seq_to_head(int S, int H, int D) {
     p.dst_head = (long long)S * D;
     p.map = MAP_FULL;
     p.T = 1;
+    set_extents(p, (long long)S * H * D, (long long)S * H * D, (long long)S * D);
     return p;
 }
 
@@ -196,6 +225,7 @@ MetricParams make_metric_params(const uint16_t *prev_v, const uint16_t *cur_v, i
     mp.sel.mask = mask;
     mp.sel.idx = idx;
     mp.sel.n_active = n_active;
+    mp.sel.debug = mp.debug = debug_counter();
     return mp;
 }
 
@@ -228,6 +258,7 @@ MoveParams make_pack_params(const uint16_t *const in[3], uint16_t *const out[3],
     p.n_active = n_active;
     p.cs = cs;
     p.eps = eps;
+    set_extents(p, (long long)S * H * D, (long long)S * H * D, (long long)S * D);
     if (in[2]) p.job[p.njobs++] = MoveJob{in[2], out[2], nullptr};
     if (in[0]) p.job[p.njobs++] = MoveJob{in[0], out[0], wq};
     if (in[1]) p.job[p.njobs++] = MoveJob{in[1], out[1], wk};
@@ -259,6 +290,7 @@ MoveParams make_unpack_params(const uint16_t *const in[3], uint16_t *const out[3
     p.n_units = S / T;
     p.idx = idx;
     p.n_active = n_active;
+    set_extents(p, (long long)S * H * D, (long long)S * H * D, 0);
     for (int i = 2; i >= 0; --i)
         if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr};
     return p;
@@ -326,6 +358,7 @@ int cocodiff_qk_norm_rope(const uint16_t *q, const uint16_t *k, uint16_t *q_out,
     p.T = 1;
     p.cs = cs;
     p.eps = eps;
+    set_extents(p, (long long)S * H * D, (long long)S * H * D, (long long)S * D);
     if (q) p.job[p.njobs++] = MoveJob{q, q_out, wq};
     if (k) p.job[p.njobs++] = MoveJob{k, k_out, wk};
     if (p.njobs == 0) return COCODIFF_OK;
@@ -366,6 +399,7 @@ int cocodiff_ulysses_a2a_inverse(const uint16_t *q_head, const uint16_t *k_head,
     p.dst_head = D;
     p.map = MAP_FULL;
     p.T = 1;
+    set_extents(p, (long long)S * H * D, (long long)S * H * D, 0);
     for (int i = 2; i >= 0; --i)
         if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr};
     if (p.njobs == 0) return COCODIFF_OK;
@@ -433,6 +467,7 @@ int cocodiff_prologue_host(const uint16_t *q_host, const uint16_t *k_host, const
         p.n_slots = len;
         p.cs = cs + (size_t)s0 * D;
         p.eps = eps;
+        set_extents(p, (long long)len * H * D, (long long)E - (long long)s0 * D, (long long)(S - s0) * D);
         for (int i = 0; i < 3; ++i) {
             CK(cudaMemcpyAsync(din[i] + s0 * tok_in, hin[i] + s0 * tok_in, (size_t)len * tok_in * 2,
                                cudaMemcpyHostToDevice, st));
@@ -474,6 +509,7 @@ int cocodiff_vmajor_select(const uint64_t *metric, int n, double r, int n_groups
     sp.mask = mask;
     sp.idx = idx;
     sp.n_active = n_active;
+    sp.debug = debug_counter();
     CK(launch_select(sp, (cudaStream_t)stream));
     return COCODIFF_OK;
 }
@@ -709,6 +745,7 @@ int cocodiff_tapa_phase1(const uint16_t *q, const uint16_t *k, const uint16_t *v
         p.src_head = p.dst_head = D;
         p.map = MAP_FULL;
         p.T = 1;
+        set_extents(p, (long long)E, (long long)E, 0);
         for (int i = 2; i >= 0; --i)
             if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i] + (size_t)t * E, nullptr};
         if (p.njobs == 0) return COCODIFF_OK;
@@ -742,6 +779,7 @@ int cocodiff_tapa_phase2(const uint16_t *q_p1, const uint16_t *k_p1, const uint1
     tp.H = H;
     tp.Hl = H / P;
     tp.heads_per_block = 8;
+    tp.debug = debug_counter();
     CK(launch_tapa_phase2(tp, D, (cudaStream_t)stream));
     return COCODIFF_OK;
 }
@@ -801,6 +839,42 @@ int cocodiff_vmajor_select_compact_static(const uint16_t *prev_v, const uint16_t
         return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, active_slots(S, T, r, n_groups), S,
                             H, D, T, st, PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
     return COCODIFF_OK;
+}
+
+long long cocodiff_debug_bounds_violations(void) {
+#ifdef COCODIFF_DEBUG_BOUNDS
+    if (!debug_counter()) return -2;
+    if (cudaDeviceSynchronize() != cudaSuccess) return -2;
+    unsigned long long count = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&count, g_bounds_violations, sizeof count) != cudaSuccess) return -2;
+    if (cudaMemcpyToSymbol(g_bounds_violations, &zero, sizeof zero) != cudaSuccess) return -2;
+    return (long long)count;
+#else
+    return -1;
+#endif
+}
+
+long long cocodiff_debug_bounds_selftest(const uint16_t *x, uint16_t *y, int S, int H, int D, void *stream) {
+#ifdef COCODIFF_DEBUG_BOUNDS
+    if (!x || !y || S < 2 || H < 1 || !supported_d(D) || !aligned16(x) || !aligned16(y)) return -2;
+    if (cocodiff_debug_bounds_violations() < 0) return -2;  // waits and clears the counter
+    // a plain [S][H][D] -> [S][H][D] move that is told its buffers end after S/2 tokens
+    MoveParams p;
+    std::memset(&p, 0, sizeof p);
+    p.n_slots = S;
+    p.H = H;
+    p.src_tok = p.dst_tok = (long long)H * D;
+    p.src_head = p.dst_head = D;
+    p.map = MAP_FULL;
+    p.T = 1;
+    set_extents(p, (long long)(S / 2) * H * D, (long long)(S / 2) * H * D, 0);
+    p.job[p.njobs++] = MoveJob{x, y, nullptr};
+    if (launch_move(p, D, (cudaStream_t)stream) != cudaSuccess) return -2;
+    return cocodiff_debug_bounds_violations();
+#else
+    (void)x; (void)y; (void)S; (void)H; (void)D; (void)stream;
+    return -1;
+#endif
 }
 
 }  // extern "C"

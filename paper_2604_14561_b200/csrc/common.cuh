@@ -24,6 +24,16 @@ enum PdlFlags : int {
     PDL_LAUNCH_ATTR = 8      // host side: launch with programmatic stream serialization
 };
 
+// Bounds-checked build (-DCOCODIFF_DEBUG_BOUNDS): every global access of the
+// kernels is checked against the extent of the buffer it belongs to; a
+// violation is counted in *debug and the access is skipped (nothing traps).
+// In the normal build the check is the constant `true` and costs nothing.
+#ifdef COCODIFF_DEBUG_BOUNDS
+#define COCODIFF_IN_BOUNDS(cond, counter) ((cond) ? true : (atomicAdd((counter), 1ull), false))
+#else
+#define COCODIFF_IN_BOUNDS(cond, counter) (true)
+#endif
+
 struct MoveJob {
     const uint16_t *src;
     uint16_t *dst;
@@ -51,6 +61,9 @@ struct MoveParams {
     int pdl;                // programmatic dependent launch: see PdlFlags
     int head_split;         // blocks per tile along the heads (>= 1); set by the launcher
     int order;              // block order; set by the launcher
+    long long src_extent, dst_extent;  // elements reachable from job.src / job.dst (bounds-checked build)
+    long long cs_extent;               // floats reachable from cs
+    unsigned long long *debug;         // violation counter (bounds-checked build), else nullptr
 };
 
 struct SelectParams {
@@ -59,6 +72,7 @@ struct SelectParams {
     uint8_t *mask;
     int32_t *idx;
     int32_t *n_active;
+    unsigned long long *debug;
 };
 
 struct MetricParams {
@@ -72,6 +86,7 @@ struct MetricParams {
     int n_units;
     SelectParams sel;
     int pdl;                      // PDL_TRIGGER: dependents may start once every block streams
+    unsigned long long *debug;
 };
 
 // Phase 2 of the two-phase exchange: up to three tensors, src = [2][S][H][D] (the
@@ -82,6 +97,7 @@ struct TapaParams {
     int n;                 // tensors
     int S, H, Hl;          // Hl = H / P heads per rank
     int heads_per_block;
+    unsigned long long *debug;
 };
 
 cudaError_t launch_tapa_phase2(const TapaParams &p, int D, cudaStream_t stream);

@@ -122,11 +122,23 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
     long long s = o, d = o;
     if (p.map != MAP_FULL) {
         const int a = o / p.T;
+        (void)COCODIFF_IN_BOUNDS(a >= 0 && a < p.n_units, p.debug);
         int unit = __ldcg(p.idx + a);  // a list that was never written must not send accesses out of bounds
         unit = unit < 0 ? 0 : (unit >= p.n_units ? p.n_units - 1 : unit);
         const long long tk = (long long)unit * p.T + (o - a * p.T);
         if (p.map == MAP_GATHER) s = tk; else d = tk;
     }
+    // bounds-checked build only: is the 16-byte vector at ptr inside its buffer?
+    auto src_ok = [&](const uint4 *ptr) {
+        return COCODIFF_IN_BOUNDS(reinterpret_cast<const uint16_t *>(ptr) >= job.src &&
+                                  reinterpret_cast<const uint16_t *>(ptr) - job.src + 8 <= p.src_extent, p.debug);
+    };
+    auto dst_ok = [&](const uint4 *ptr) {
+        return COCODIFF_IN_BOUNDS(reinterpret_cast<const uint16_t *>(ptr) >= job.dst &&
+                                  reinterpret_cast<const uint16_t *>(ptr) - job.dst + 8 <= p.dst_extent, p.debug);
+    };
+    (void)src_ok;
+    (void)dst_ok;
     const uint4 *sp = reinterpret_cast<const uint4 *>(job.src + s * p.src_tok) + lr + h_lo * sh;
     uint4 *dp = reinterpret_cast<uint4 *>(job.dst + d * p.dst_tok) + lr + h_lo * dh;
 
@@ -137,9 +149,9 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
             constexpr int U = decltype(u_tag)::value;
             uint4 v[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) { v[u] = ld_row<HINT>(sp); sp += sh; }
+            for (int u = 0; u < U; ++u) { v[u] = src_ok(sp) ? ld_row<HINT>(sp) : make_uint4(0, 0, 0, 0); sp += sh; }
 #pragma unroll
-            for (int u = 0; u < U; ++u) { st_row<HINT>(dp, v[u]); dp += dh; }
+            for (int u = 0; u < U; ++u) { if (dst_ok(dp)) st_row<HINT>(dp, v[u]); dp += dh; }
         });
         return;
     }
@@ -157,7 +169,9 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
         if (p.cs != nullptr) {
             // pairs 4*lr .. 4*lr+3 of token s: 8 floats (cos, sin, cos, sin, ...)
             const float4 *tb = reinterpret_cast<const float4 *>(p.cs + s * D) + 2 * lr;
-            const float4 t0 = __ldg(tb), t1 = __ldg(tb + 1);
+            const bool cs_ok = COCODIFF_IN_BOUNDS(s >= 0 && s * D + 8 * lr + 8 <= p.cs_extent, p.debug);
+            const float4 t0 = cs_ok ? __ldg(tb) : make_float4(1.f, 0.f, 1.f, 0.f);
+            const float4 t1 = cs_ok ? __ldg(tb + 1) : make_float4(1.f, 0.f, 1.f, 0.f);
             c[0] = t0.x; sn[0] = t0.y; c[1] = t0.z; sn[1] = t0.w;
             c[2] = t1.x; sn[2] = t1.y; c[3] = t1.z; sn[3] = t1.w;
         }
@@ -198,11 +212,11 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
         constexpr int U = decltype(u_tag)::value;
         uint4 v[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) { v[u] = ld_row<HINT>(sp); sp += sh; }
+        for (int u = 0; u < U; ++u) { v[u] = src_ok(sp) ? ld_row<HINT>(sp) : make_uint4(0, 0, 0, 0); sp += sh; }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const uint4 y = norm_rope_row(v[u]);
-            if (valid) st_row<HINT>(dp, y);
+            if (valid && dst_ok(dp)) st_row<HINT>(dp, y);
             dp += dh;
         }
     });

@@ -38,13 +38,18 @@ __global__ void __launch_bounds__(kThreads) tapa_phase2_kernel(const __grid_cons
             const int h = h0 + u;
             if (h < h_hi) {
                 const int ring = (h / p.Hl) & 1;  // destination rank r = h / Hl sits on ring r % 2
-                v[u] = __ldcs(reinterpret_cast<const uint4 *>(src + ring * E + ((long long)s * p.H + h) * D) + lr);
+                const long long off = ring * E + ((long long)s * p.H + h) * D + 8 * lr;
+                v[u] = COCODIFF_IN_BOUNDS(off >= 0 && off + 8 <= 2 * E, p.debug)
+                           ? __ldcs(reinterpret_cast<const uint4 *>(src + off)) : make_uint4(0, 0, 0, 0);
             }
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int h = h0 + u;
-            if (h < h_hi) __stcs(reinterpret_cast<uint4 *>(dst + ((long long)h * p.S + s) * D) + lr, v[u]);
+            if (h < h_hi) {
+                const long long off = ((long long)h * p.S + s) * D + 8 * lr;
+                if (COCODIFF_IN_BOUNDS(off >= 0 && off + 8 <= E, p.debug)) __stcs(reinterpret_cast<uint4 *>(dst + off), v[u]);
+            }
         }
     }
 }

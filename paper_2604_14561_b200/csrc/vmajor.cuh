@@ -107,8 +107,11 @@ __device__ void emit_selection(const SelectParams &p, int grp, const unsigned lo
         const bool tie = !none && v == mstar;
         const bool cached = !none && (v < mstar || (tie && tie_rank < t_c));
         tie_rank += tie;
-        p.mask[base + e] = cached ? 0 : 1;
-        if (!cached) p.idx[out_base + pos++] = base + e;
+        if (COCODIFF_IN_BOUNDS(base + e >= 0 && base + e < p.n, p.debug)) p.mask[base + e] = cached ? 0 : 1;
+        if (!cached) {
+            if (COCODIFF_IN_BOUNDS(out_base + pos >= 0 && out_base + pos < p.n, p.debug)) p.idx[out_base + pos] = base + e;
+            ++pos;
+        }
     }
     if (grp == 0 && tid == 0) *p.n_active = p.n_groups * (g - p.n_cached);
     __syncthreads();
@@ -229,14 +232,18 @@ __device__ __forceinline__ void metric_stream(const MetricParams &p, const unsig
             uint4 a[U], b[U];
 #pragma unroll
             for (int i = 0; i < U; ++i)
-                if (v + 32 * i < v1) { a[i] = __ldcs(pc + v + 32 * i); b[i] = __ldcs(pp + v + 32 * i); }
+                if (v + 32 * i < v1) {
+                    const bool ok = COCODIFF_IN_BOUNDS((long long)u * p.unit_vecs + v + 32 * i < (long long)p.n_units * p.unit_vecs, p.debug);
+                    a[i] = ok ? __ldcs(pc + v + 32 * i) : make_uint4(0, 0, 0, 0);
+                    b[i] = ok ? __ldcs(pp + v + 32 * i) : make_uint4(0, 0, 0, 0);
+                }
 #pragma unroll
             for (int i = 0; i < U; ++i)
                 if (v + 32 * i < v1) acc += l1_of_vec(a[i], b[i]);
         }
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (lane == 0 && acc != 0) atomicAdd(p.acc + u, acc);
+        if (lane == 0 && acc != 0 && COCODIFF_IN_BOUNDS(u < (unsigned)p.n_units, p.debug)) atomicAdd(p.acc + u, acc);
     }
 }
 
