@@ -87,7 +87,7 @@ cudaError_t launch_select(const SelectParams &p, cudaStream_t stream, int pdl) {
         return launch_maybe_programmatic(vmajor_select_small_kernel, dim3(p.n_groups), dim3(256), 0, stream, pdl, p, pdl);
     // stage the group's metrics in shared memory when they fit beside the histograms
     const size_t want = (size_t)p.g * sizeof(unsigned long long);
-    const size_t limit = 160 * 1024;
+    const size_t limit = 188 * 1024;  // with the 37 KB of static shared memory: inside the 227 KB a block may use
     const int staged = want <= limit ? 1 : 0;
     const size_t dyn = staged ? want : 0;
     static bool attr_set[64] = {};
