@@ -185,9 +185,10 @@ int cocodiff_unpack_qkv(const uint16_t *q_compact, const uint16_t *k_compact, co
  * metric and selection on V, compaction of the active units of V (moved) and of
  * Q, K (normalised and rotated on the way), then - if the three caches are
  * given - the scatter over the cached HEAD tensors.  V_FIRST with two streams:
- * metric, selection and V's compaction run on stream_v, Q and K start on
- * stream_qk as soon as the index list exists; LUMP or equal streams: one stream,
- * the three compactions in one launch.  Stream semantics as for
+ * metric, selection and V's compaction run on stream_v, Q and K follow on
+ * stream_qk when V's part is done; LUMP or equal streams: one stream, the three
+ * compactions in one launch.  Consecutive kernels of a stream are chained with
+ * programmatic dependent launches.  Stream semantics as for
  * cocodiff_ulysses_a2a; outputs and workspace as for
  * cocodiff_vmajor_select_compact.  The caches are all given or all NULL. */
 int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const uint16_t *k, const uint16_t *v,

@@ -649,27 +649,29 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
         if (rc) return rc;
         unpack_pdl = PDL_LAUNCH_ATTR | PDL_WAIT_AT_START;
     } else {
-        // V first: metric, selection and V's compaction on stream_v; Q and K follow on
-        // stream_qk as soon as the index list exists.
+        // V first: metric, selection and V's compaction on stream_v, chained with dependent
+        // launches; Q and K follow on stream_qk once V's part is done, and the scatter is
+        // chained behind their compaction.
         ForkJoin *fj = nullptr;
         rc = get_events(&fj);
         if (rc) return rc;
         CK(cudaEventRecord(fj->fork, sq));
         CK(cudaStreamWaitEvent(sv, fj->fork, 0));
-        rc = enqueue_metric_select(prev_v, v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, sv);
+        rc = enqueue_metric_select(prev_v, v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, sv,
+                                   PDL_TRIGGER);
         if (rc) return rc;
-        CK(cudaEventRecord(fj->fork, sv));
-        CK(cudaStreamWaitEvent(sq, fj->fork, 0));
         const uint16_t *in_v[3] = {nullptr, nullptr, v};
         uint16_t *out_v[3] = {nullptr, nullptr, v_compact};
-        rc = enqueue_pack(in_v, out_v, nullptr, nullptr, 0.f, nullptr, idx, n_active, slots, S, H, D, T, sv);
-        if (rc) return rc;
-        const uint16_t *in_qk[3] = {q, k, nullptr};
-        uint16_t *out_qk[3] = {q_compact, k_compact, nullptr};
-        rc = enqueue_pack(in_qk, out_qk, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T, sq);
+        rc = enqueue_pack(in_v, out_v, nullptr, nullptr, 0.f, nullptr, idx, n_active, slots, S, H, D, T, sv,
+                          PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
         if (rc) return rc;
         CK(cudaEventRecord(fj->join, sv));
         CK(cudaStreamWaitEvent(sq, fj->join, 0));
+        const uint16_t *in_qk[3] = {q, k, nullptr};
+        uint16_t *out_qk[3] = {q_compact, k_compact, nullptr};
+        rc = enqueue_pack(in_qk, out_qk, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T, sq, PDL_TRIGGER);
+        if (rc) return rc;
+        unpack_pdl = PDL_LAUNCH_ATTR | PDL_WAIT_AT_START;
     }
     if (do_unpack) return enqueue_unpack(comp_in, cache, idx, n_active, slots, S, H, D, T, sq, unpack_pdl);
     return COCODIFF_OK;
