@@ -132,7 +132,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
         "us_per_layer_extrapolated": 1e6 * total / args.steps * cfg["S"] / tokens,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 storage, fp32 arithmetic",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "storage_dtype": "bf16",
         "data": "synthetic", "config": {"workload": WORKLOAD, "P": cfg["P"], "S": cfg["S"], "H": cfg["H"],
                                         "D": cfg["D"], "sample": sample},
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
@@ -382,7 +382,7 @@ def run_ours(args):
             "frac_of_nominal_8000": value / world / NOMINAL_HBM_GBS, "frac_of_measured_copy": value / world / peak,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16 storage, fp32 arithmetic", "data": "synthetic",
+            "dtype": "f32", "storage_dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "P": P, "S": S, "H": H, "D": D, "order": "v_first",
                        "algorithmic_bytes_per_step": step_bytes, "l2": "inputs and outputs (775 MB per step) exceed the 126 MB L2",
                        "replicas": world},
