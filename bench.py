@@ -361,6 +361,7 @@ def run_ours(args):
         del hin, hout, dev_in, dev_out
 
         per_config = other_configs(torch, binding, args)
+        per_config["next_rows_temporal"] = next_rows(torch, binding, args)
 
         # ---- the oracle on this machine's host cores, bounded sample ------------
         import oracle
@@ -509,6 +510,103 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
     return out
 
 
+def next_rows(torch, binding, args):
+    """Rows beyond the headline path, on the temporal workload (P=24, S=9216, H=24, D=128):
+    inverse exchange, the two TAPA phases, per-token selection units, and the paper's
+    50-step cache schedule (5 warm-up steps, refresh every 10 steps, linear cache ratio)."""
+    cfg = synth.config("temporal")
+    P, S, H, D = cfg["P"], cfg["S"], cfg["H"], cfg["D"]
+    E = S * H * D
+    L = synth.make_layer(cfg)
+    q, k, v = (dev(L[n], torch) for n in "qkv")
+    wq, wk = dev(L["wq"], torch), dev(L["wk"], torch)
+    cs = torch.empty((S, D // 2, 2), dtype=torch.float32, device="cuda")
+    binding.rope_table_2d(cs, dev(L["pos"], torch), S, D, cfg["theta"])
+    new = lambda n=1: torch.empty(n * E, dtype=torch.int16, device="cuda")
+    qh, kh, vh = new(), new(), new()
+    scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    sink = torch.zeros(1, dtype=torch.int64, device="cuda")
+    sq, sv = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def flush():
+        with torch.cuda.stream(sq):
+            scratch.zero_()
+            torch.sum(scratch.view(torch.int64), dim=0, keepdim=True, out=sink)
+
+    iters = max(10, min(args.steps, 30))
+    out = {}
+
+    def timed(name, fn, nbytes):
+        t = statistics.median(time_steps(torch, fn, sq, iters, 3, flush=flush))
+        out[name] = {"us_cold_l2": 1e3 * t, "bytes": nbytes, "gbs": nbytes / (t * 1e-3) / 1e9}
+
+    binding.prologue(q, k, v, qh, kh, vh, wq, wk, cfg["eps"], cs, P, S, H, D, order=binding.LUMP, stream_qk=sq, stream_v=sq)
+    back = [new() for _ in range(3)]
+    timed("inverse_a2a", lambda: binding.ulysses_a2a_inverse(qh, kh, vh, *back, P, S, H, D, stream=sq), 6 * E * 2)
+    del back
+    p1 = [new(2) for _ in range(3)]
+    th = [new() for _ in range(3)]
+    timed("tapa_phase1", lambda: binding.tapa_phase1(q, k, v, *p1, P, S, H, D, stream=sq), 12 * E * 2)
+    timed("tapa_phase2", lambda: binding.tapa_phase2(*p1, *th, P, S, H, D, stream=sq), 6 * E * 2)
+    del p1, th
+
+    # per-token selection units (T = 1): 20 % of the tokens changed strongly
+    comp = [new() for _ in range(3)]
+    for T, label in ((1, "selective_step_T1"),):
+        n = S // T
+        rng = np.random.default_rng(0)
+        hot = np.sort(rng.choice(n, int(np.ceil(0.2 * n)), replace=False))
+        cur = synth.bf16_bits_to_f32(L["v"]).reshape(n, -1).copy()
+        cur[hot] += 0.5
+        cur_v = dev(synth.f32_to_bf16_bits(cur).reshape(S, H, D), torch)
+        ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        metric = torch.zeros(n, dtype=torch.int64, device="cuda")
+        mask = torch.zeros(n, dtype=torch.uint8, device="cuda")
+        idx = torch.zeros(n, dtype=torch.int32, device="cuda")
+        na = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for groups in (1, P):
+            def step():
+                binding.selective_prologue(v, q, k, cur_v, wq, wk, cfg["eps"], cs, P, S, H, D, T, 0.8, groups, metric,
+                                           mask, idx, na, comp[0], comp[1], comp[2], qh, kh, vh, ws, ws_bytes,
+                                           order=binding.LUMP, stream_qk=sq, stream_v=sq)
+            t = statistics.median(time_steps(torch, step, sq, iters, 3, flush=flush))
+            n_act = int(na.item())
+            nbytes = 2 * E * 2 + 12 * n_act * T * H * D * 2
+            out[f"{label}_groups{groups}"] = {"us_cold_l2": 1e3 * t, "n_units": n, "n_active": n_act, "bytes": nbytes,
+                                              "gbs": nbytes / (t * 1e-3) / 1e9}
+
+    # the 50-step schedule on 64-token tiles, inputs fixed (timing only), back to back
+    T, total, warmup, interval = cfg["T"], 50, 5, 10
+    n = S // T
+    ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    metric = torch.zeros(n, dtype=torch.int64, device="cuda")
+    mask = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    idx = torch.zeros(n, dtype=torch.int32, device="cuda")
+    na = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(total + 1)]
+    for rep in range(2):                 # first pass warms up
+        sent = []
+        torch.cuda.synchronize()
+        ev[0].record(sq)
+        for step_i in range(total):
+            _, s_el = binding.layer_step(step_i, total, warmup, interval, v, q, k, v, wq, wk,
+                                         cfg["eps"], cs, P, S, H, D, T, 1, metric, mask, idx, na, comp[0], comp[1],
+                                         comp[2], qh, kh, vh, ws, ws_bytes, order=binding.LUMP, stream_qk=sq, stream_v=sq)
+            sent.append(s_el)
+            ev[step_i + 1].record(sq)
+        torch.cuda.synchronize()
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(total)]
+    full = [binding.cache_schedule(i, total, warmup, interval)[0] for i in range(total)]
+    out["schedule_50_steps"] = {
+        "total_us": 1e3 * sum(per_step), "always_full_us_estimate": 1e3 * total * statistics.mean(t for t, f in zip(per_step, full) if f),
+        "full_steps": sum(full), "us_full_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if f),
+        "us_selective_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if not f),
+        "exchanged_fraction_of_always_full": sum(sent) / (total * 3 * E), "l2": "warm (steps back to back)"}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -526,7 +624,9 @@ def main():
         import torch
         from paper_2604_14561_b200 import binding
         torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-        print(json.dumps({"per_config": other_configs(torch, binding, args, names=("temporal",))}, ensure_ascii=False))
+        pc = other_configs(torch, binding, args, names=("temporal",))
+        pc["next_rows_temporal"] = next_rows(torch, binding, args)
+        print(json.dumps({"per_config": pc}, ensure_ascii=False))
     else:
         run_ours(args)
 
