@@ -239,7 +239,7 @@ int oracle_ulysses_a2a_inverse(const uint16_t *head, uint16_t *seq, int P, int S
 /* Tile-aware parallel all-to-all (TAPA, Section III-B).  Ranks 2g and 2g+1    */
 /* are the two tiles of GPU g; P must be even.                                 */
 /* Phase 1: inside every GPU the two tiles swap their whole shards (S/P tokens,*/
-/* all heads - the "14 MB message" of the running example for Q, K, V), so     */
+/* all heads - 14 MB for Q, K, V together in the running example), so         */
 /* that afterwards each tile holds all tokens of its GPU in token order.       */
 /* p1 layout: [2][P/2][2*S/P][H][D], p1[t][g] = what tile t of GPU g holds.    */
 /* With this layout p1[t] as a whole is again a [S][H][D] tensor.              */

@@ -147,5 +147,5 @@ def test_tapa_needs_an_even_rank_count_and_its_message_is_the_whole_shard():
         oracle.tapa_phase1(_rand_bits((9, 3, 4), 23), 3)
     g = _golden()
     P, S, H, D = map(int, g["phase1_message_mb"][0].split())
-    # a tile sends its S/P tokens with all heads, for Q, K and V: "each message is 14 MB"
+    # a tile sends its S/P tokens with all heads, for Q, K and V: the 14 MB message size of Section III-B
     assert round(3 * (S // P) * H * D * 2 / 1e6) == g["phase1_message_mb"][2]
