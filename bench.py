@@ -93,16 +93,52 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------- CPU oracle ---
-def oracle_sample(cfg, L, tokens):
-    """The oracle's full prologue on the first `tokens` tokens of the layer."""
+def oracle_sample(cfg, L, tokens, keep=False):
+    """The oracle's full prologue on the first `tokens` tokens of the layer; returns the
+    seconds it took (and, with keep, its three outputs)."""
     import oracle
     P, D = cfg["P"], cfg["D"]
     sl = slice(0, tokens)
     cs = oracle.rope_table_2d(L["pos"][sl], D, cfg["theta"])
     q, k, v = (np.ascontiguousarray(L[n][sl]) for n in "qkv")
     t0 = time.perf_counter()
-    oracle.prologue(q, k, v, L["wq"], L["wk"], cfg["eps"], cs, P)
-    return time.perf_counter() - t0
+    out = oracle.prologue(q, k, v, L["wq"], L["wk"], cfg["eps"], cs, P)
+    dt = time.perf_counter() - t0
+    return (dt, out) if keep else dt
+
+
+def oracle_all_cores(sub, L, tokens, budget_s=5.0):
+    """The same oracle source built with OpenMP, on every core this process may use."""
+    import oracle
+    cores = len(os.sched_getaffinity(0))
+    try:
+        oracle.use_all_cores(True)
+        oracle_sample(sub, L, tokens)
+        reps, spent = 0, 0.0
+        while spent < budget_s and reps < 200:
+            spent += oracle_sample(sub, L, tokens)
+            reps += 1
+    finally:
+        oracle.use_all_cores(False)
+    return {"value": algorithmic_bytes(sub) * reps / spent / 1e9, "unit": "GB/s", "cores": cores,
+            "build": "the same oracle source compiled with -fopenmp", "passes": reps}
+
+
+def parity_of_sample(cfg, L, tokens, got_heads, oracle_heads):
+    """Distance statistics between the kernels' Q and K and the oracle's on the sample the
+    CPU baseline ran on (computed outside every timed region, with the tests' own rule)."""
+    import oracle
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from helpers import parity_stats
+    sl = slice(0, tokens)
+    cs = oracle.rope_table_2d(L["pos"][sl], cfg["D"], cfg["theta"])
+    out = {"tokens": tokens, "rule": "|gpu - ref| <= 2 bf16 ulp at max(|ref|, 2^-9 * magnitude of the rotated pair); "
+                                    "n_strict_fail counts elements beyond 2 ulp of their own magnitude (no floor)"}
+    for name, w, got, ref in (("q", L["wq"], got_heads[0], oracle_heads[0]), ("k", L["wk"], got_heads[1], oracle_heads[1])):
+        _, ref_f = oracle.norm_rope(np.ascontiguousarray(L[name][sl]), w, cfg["eps"], cs, want_f32=True)
+        out[name] = parity_stats(got, ref, np.ascontiguousarray(ref_f.transpose(1, 0, 2)))
+    out["v_bit_exact"] = bool(np.array_equal(got_heads[2], oracle_heads[2]))
+    return out
 
 
 def run_reference(args):
@@ -295,6 +331,20 @@ def run_ours(args):
     total_ms = max_over_ranks(total_ms, world, "cuda")
     ms_per_step = total_ms / args.steps
     value = aggregate_gbs(step_bytes, world, ms_per_step)
+    # the same back-to-back loop five more times, each at least 20 ms long whatever --steps says
+    rep_steps = max(args.steps, int(np.ceil(20.0 / ms_per_step)))
+    rep_ms = []
+    for _ in range(5):
+        barrier()
+        start.record(sq)
+        for _ in range(rep_steps):
+            step(binding.V_FIRST)
+        stop.record(sq)
+        barrier()
+        rep_ms.append(max_over_ranks(start.elapsed_time(stop), world, "cuda") / rep_steps)
+    repeats = {"n": 5, "steps_each": rep_steps, "us_per_layer_median": 1e3 * statistics.median(rep_ms),
+               "us_per_layer_min": 1e3 * min(rep_ms), "us_per_layer_max": 1e3 * max(rep_ms),
+               "gbs_median": aggregate_gbs(step_bytes, world, statistics.median(rep_ms))}
 
     line = None
     if rank == 0 and args.only_main:
@@ -342,7 +392,9 @@ def run_ours(args):
                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                     "frac": achieved / peak, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                     "us_per_launch": 1e3 * qk_ms, "algorithmic_bytes_per_launch": qk_bytes,
-                    "traffic": read_traffic_note()}
+                    "traffic": read_traffic_note(),
+                    "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel on this "
+                                      "workload, read from profiles/move_rows_kernel_qwen2304.md (not measured in this run)"}
 
         # ---- end to end: host buffers in, host buffers out ------------------
         hin = [torch.from_numpy(L[n].view(np.int16)).pin_memory() for n in "qkv"]
@@ -361,6 +413,7 @@ def run_ours(args):
         del hin, hout, dev_in, dev_out
 
         per_config = other_configs(torch, binding, args)
+        per_config["temporal_steps"] = temporal_rows(torch, binding, args)
         per_config["next_rows_temporal"] = next_rows(torch, binding, args)
 
         # ---- the oracle on this machine's host cores, bounded sample ------------
@@ -368,15 +421,20 @@ def run_ours(args):
         oracle.build()
         tokens = S // P
         sub = dict(cfg, S=tokens)
-        oracle_sample(sub, L, tokens)                       # warm the page cache / allocator
+        _, oracle_heads = oracle_sample(sub, L, tokens, keep=True)     # also warms the page cache / allocator
         reps, spent = 0, 0.0
         while spent < 10.0 and reps < 40:
             spent += oracle_sample(sub, L, tokens)
             reps += 1
         cpu_gbs = algorithmic_bytes(sub) * reps / spent / 1e9
+        step(binding.V_FIRST)
+        torch.cuda.synchronize()
+        got_heads = [t.view(H, S, D)[:, :tokens].contiguous().cpu().numpy().view(np.uint16) for t in (qh, kh, vh)]
         cpu = {"value": cpu_gbs, "unit": "GB/s", "cores": 1, "kind": "oracle",
                "ms_per_layer_extrapolated": 1e3 * spent / reps * S / tokens,
-               "sample": f"{reps} passes over the first {tokens} of {S} tokens (one rank's shard) of the same layer"}
+               "sample": f"{reps} passes over the first {tokens} of {S} tokens (one rank's shard) of the same layer",
+               "all_cores": oracle_all_cores(sub, L, tokens),
+               "parity_on_sample": parity_of_sample(cfg, L, tokens, got_heads, oracle_heads)}
 
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "us_per_layer": 1e3 * ms_per_step,
@@ -388,6 +446,7 @@ def run_ours(args):
                        "algorithmic_bytes_per_step": step_bytes, "l2": "inputs and outputs (775 MB per step) exceed the 126 MB L2",
                        "replicas": world},
             "gpu_launches": 2 * args.steps,
+            "repeats": repeats,
             "clocks": clocks, "orders": orders, "v_first_timeline": v_first_timeline, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
             "per_config": per_config,
         }
@@ -410,25 +469,48 @@ def read_traffic_note():
         return None
 
 
+class Flusher:
+    """Between timed iterations: write a buffer four times the L2, then read it back.  The L2
+    ends up full of clean foreign lines, so the timed region neither hits in L2 nor pays for
+    the write-back of the flush's own dirty lines."""
+
+    def __init__(self, torch, stream):
+        self.torch, self.stream = torch, stream
+        self.scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+        self.sink = torch.zeros(1, dtype=torch.int64, device="cuda")
+
+    def __call__(self):
+        with self.torch.cuda.stream(self.stream):
+            self.scratch.zero_()
+            self.torch.sum(self.scratch.view(self.torch.int64), dim=0, keepdim=True, out=self.sink)
+
+
+def launch_floor(torch, binding, sq, flush, iters):
+    """What one launch costs between two events, whatever it moves: the same prologue call on
+    16 tokens of one head (8 KB), timed with the same protocol as the small workloads."""
+    S, H, D = 16, 1, 128
+    x = [torch.zeros(S * H * D, dtype=torch.int16, device="cuda") for _ in range(6)]
+    w = torch.full((D,), 0x3F80, dtype=torch.int16, device="cuda")
+    cs = torch.zeros((S, D // 2, 2), dtype=torch.float32, device="cuda")
+    cs[..., 0] = 1.0
+
+    def call():
+        binding.prologue(x[0], x[1], x[2], x[3], x[4], x[5], w, w, 1e-6, cs, 1, S, H, D, order=binding.LUMP,
+                         stream_qk=sq, stream_v=sq)
+    return 1e3 * statistics.median(time_steps(torch, call, sq, iters, 3, flush=flush))
+
+
 def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "temporal")):
-    """µs/layer and GB/s of the other synthetic workloads, L2 flushed between
-    iterations (they fit in the 126 MB L2; flush = write then read 512 MB), plus the selective step of the
-    temporal workload."""
+    """µs/layer of the other synthetic workloads, L2 flushed between iterations.  They fit in
+    the 126 MB L2, so part of their output is still dirty in the L2 when the timed region ends:
+    the GB/s given for them is effective throughput (algorithmic bytes / time), not HBM traffic."""
     out = {}
-    scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
     sq, sv = torch.cuda.Stream(), torch.cuda.Stream()
-
-    sink = torch.zeros(1, dtype=torch.int64, device="cuda")
-
-    def flush():
-        # write a buffer four times the L2, then read it back: the L2 ends up full of
-        # clean lines, so the timed region neither hits in L2 nor pays for the write-back
-        # of the flush's own dirty lines
-        with torch.cuda.stream(sq):
-            scratch.zero_()
-            torch.sum(scratch.view(torch.int64), dim=0, keepdim=True, out=sink)
-
+    flush = Flusher(torch, sq)
     iters = max(10, min(args.steps, 50))
+    floor = launch_floor(torch, binding, sq, flush, iters)
+    out["launch_floor"] = {"us": floor, "what": "median event-to-event time of one prologue launch that moves 8 KB, same "
+                                                "flush-and-events protocol: the fixed cost inside every per_config figure"}
     for name in names:
         cfg = synth.config(name)
         P, S, H, D = cfg["P"], cfg["S"], cfg["H"], cfg["D"]
@@ -444,76 +526,108 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
             binding.prologue(q, k, v, qh, kh, vh, wq, wk, cfg["eps"], cs, P, S, H, D,
                              order=order, stream_qk=sq, stream_v=sv)
         b = algorithmic_bytes(cfg)
-        out[name] = {"bytes": b}
+        out[name] = {"bytes": b, "fits_in_l2": b < 126e6 * 2}
         for oname, order in (("v_first", binding.V_FIRST), ("lump", binding.LUMP)):
             cold = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 3, flush=flush))
             warm = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 3))
-            out[name][oname] = {"us_cold_l2": 1e3 * cold, "gbs_cold_l2": b / (cold * 1e-3) / 1e9,
+            out[name][oname] = {"us_cold_l2": 1e3 * cold, "gbs_effective_cold_l2": b / (cold * 1e-3) / 1e9,
+                                "gbs_effective_above_launch_floor": b / max(1e3 * cold - floor, 1e-3) / 1e3,
                                 "us_warm_l2": 1e3 * warm}
             gr = time_graph(torch, lambda: full(order), sq, iters, flush=flush)
             if gr is not None:
                 out[name][oname]["us_cold_l2_cuda_graph"] = 1e3 * statistics.median(gr)
-        if name != "temporal":
-            continue
-        # selective step: metric + selection + V compaction, K/Q compaction (norm + RoPE fused), three scatters
-        T, r, n_groups = cfg["T"], cfg["r"], cfg["n_groups"]
-        n = S // T
-        seq_rng = np.random.default_rng(0)
-        hot = np.sort(seq_rng.choice(n, int(np.ceil(cfg["frac_large"] * n)), replace=False))
-        cur = synth.bf16_bits_to_f32(L["v"]).reshape(n, -1).copy()
-        cur[hot] += synth.normal_f32(9, "bump", len(hot) * cur.shape[1], 0.0, cfg["sigma_large"]).reshape(len(hot), -1)
-        cur_v = dev(synth.f32_to_bf16_bits(cur).reshape(S, H, D), torch)
-        ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
-        ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
-        metric = torch.zeros(n, dtype=torch.int64, device="cuda")
-        mask = torch.zeros(n, dtype=torch.uint8, device="cuda")
-        idx = torch.zeros(n, dtype=torch.int32, device="cuda")
-        na = torch.zeros(1, dtype=torch.int32, device="cuda")
-        comp = [torch.empty(E, dtype=torch.int16, device="cuda") for _ in range(3)]
+        del q, k, v, qh, kh, vh
+    return out
 
-        def selective(order):
-            binding.selective_prologue(v, q, k, cur_v, wq, wk, cfg["eps"], cs, P, S, H, D, T, r, n_groups,
-                                       metric, mask, idx, na, comp[0], comp[1], comp[2], qh, kh, vh,
-                                       ws, ws_bytes, order=order, stream_qk=sq, stream_v=sv)
-        sel = {}
-        for oname, order in (("lump", binding.LUMP), ("v_first", binding.V_FIRST)):
-            cold = time_steps(torch, lambda: selective(order), sq, iters, 3, flush=flush)
-            sel[oname] = 1e3 * statistics.median(cold)
-            gr = time_graph(torch, lambda: selective(order), sq, iters, flush=flush)
-            if gr is not None:
-                sel[oname + "_cuda_graph"] = 1e3 * statistics.median(gr)
-        n_act = int(na.item())
-        tile = T * H * D * 2
-        sb = 2 * E * 2 + 3 * 2 * n_act * tile + 3 * 2 * n_act * tile
 
-        def part_select():
-            binding.vmajor_select_compact(v, cur_v, P, S, H, D, T, r, n_groups, metric, mask, idx, na, None,
-                                          ws, ws_bytes, stream=sq)
+def temporal_rows(torch, binding, args):
+    """The temporal workload as its eight denoising steps (step t+1 = step t + N(0, 1e-3)
+    everywhere + N(0, 0.5) on a fifth of the 64-token tiles, re-drawn every step): step 0 is a
+    full exchange that fills the caches, steps 1-7 are selective steps at r = 0.8 against
+    prev_v = V of the step before.  Every step is timed on its own (cold L2, median)."""
+    cfg = synth.config("temporal")
+    P, S, H, D, T, r, n_groups = cfg["P"], cfg["S"], cfg["H"], cfg["D"], cfg["T"], cfg["r"], cfg["n_groups"]
+    E, n = S * H * D, S // T
+    seq = synth.TemporalSequence(cfg)
+    steps = []
+    for t in range(cfg["steps"]):
+        if t:
+            seq.advance()
+        cur = seq.current()
+        steps.append({x: dev(cur[x], torch) for x in "qkv"})
+    wq, wk = dev(seq.wq, torch), dev(seq.wk, torch)
+    cs = torch.empty((S, D // 2, 2), dtype=torch.float32, device="cuda")
+    binding.rope_table_2d(cs, dev(seq.pos, torch), S, D, cfg["theta"])
+    new = lambda: torch.empty(E, dtype=torch.int16, device="cuda")
+    cache, comp = [new() for _ in range(3)], [new() for _ in range(3)]
+    ws = torch.empty(1 << 20, dtype=torch.uint8, device="cuda")
+    metric = torch.zeros(S, dtype=torch.int64, device="cuda")
+    mask = torch.zeros(S, dtype=torch.uint8, device="cuda")
+    idx = torch.zeros(S, dtype=torch.int32, device="cuda")
+    na = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sq, sv = torch.cuda.Stream(), torch.cuda.Stream()
+    flush = Flusher(torch, sq)
+    iters = max(10, min(args.steps, 30))
+    tile = T * H * D * 2
 
-        def part_pack():
-            binding.pack_active_qkv(q, k, cur_v, wq, wk, cfg["eps"], cs, idx, na, comp[0], comp[1], comp[2],
-                                    P, S, H, D, T, stream=sq)
+    def full_step(order):
+        x = steps[0]
+        binding.prologue(x["q"], x["k"], x["v"], *cache, wq, wk, cfg["eps"], cs, P, S, H, D, order=order,
+                         stream_qk=sq, stream_v=sv)
 
-        def part_unpack():
-            binding.unpack_qkv(comp[0], comp[1], comp[2], idx, na, qh, kh, vh, P, S, H, D, T, stream=sq)
-        breakdown = {}
-        for pname, fn, nbytes in (("metric_select", part_select, 2 * E * 2), ("pack_qkv", part_pack, 6 * n_act * tile),
-                                  ("unpack_qkv", part_unpack, 6 * n_act * tile)):
-            t = statistics.median(time_steps(torch, fn, sq, iters, 3, flush=flush))
-            breakdown[pname] = {"us_cold_l2": 1e3 * t, "bytes": nbytes, "gbs": nbytes / (t * 1e-3) / 1e9}
-        best = min(sel.values())
-        out["temporal_selective_step"] = {"n_active": n_act, "n_units": n, "bytes": sb,
-                                          "us_cold_l2": sel, "gbs_cold_l2_best": sb / (best * 1e-6) / 1e9,
-                                          "launches_per_step": {"lump": 4, "v_first": 5},
-                                          "parts_timed_alone": breakdown,
-                                          "api": "cocodiff_selective_prologue"}
+    def selective(t, order, T_=T, groups=n_groups):
+        x, prev = steps[t], steps[t - 1]["v"]
+        binding.selective_prologue(prev, x["q"], x["k"], x["v"], wq, wk, cfg["eps"], cs, P, S, H, D, T_, r, groups,
+                                   metric, mask, idx, na, *comp, *cache,
+                                   ws, binding.vmajor_workspace_bytes(P, S, H, D, T_), order=order,
+                                   stream_qk=sq, stream_v=sv if order == binding.V_FIRST else sq)
+    out = {"workload": "temporal: P=24, S=9216, H=24, D=128, T=64, r=0.8, one global group; 8 steps of the data law",
+           "l2": "flushed (write + read of 512 MB) before every timed call"}
+    fb = 6 * E * 2
+    t_full = {o: 1e3 * statistics.median(time_steps(torch, lambda: full_step(order), sq, iters, 3, flush=flush))
+              for o, order in (("v_first", binding.V_FIRST), ("lump", binding.LUMP))}
+    out["step_0_full"] = {"us_cold_l2": t_full, "bytes": fb, "gbs_best": fb / (min(t_full.values()) * 1e-6) / 1e9}
+    per_step = []
+    for t in range(1, cfg["steps"]):
+        row = {"step": t}
+        for o, order in (("lump", binding.LUMP), ("v_first", binding.V_FIRST)):
+            row["us_" + o] = 1e3 * statistics.median(time_steps(torch, lambda: selective(t, order), sq, iters, 3, flush=flush))
+        row["n_active"] = int(na.item())
+        per_step.append(row)
+    n_act = per_step[0]["n_active"]
+    b_alg = 2 * E * 2 + 12 * n_act * tile          # metric pass + compaction (read, write) + scatter (read, write)
+    b_moved = 2 * E * 2 + 9 * n_act * tile         # gather and scatter in one pass: one read, two writes per active row
+    mean = {o: statistics.mean(row["us_" + o] for row in per_step) for o in ("lump", "v_first")}
+    best = min(mean.values())
+    peak, _ = measured_peak()
+    out["steps_1_to_7_selective"] = {
+        "per_step": per_step, "us_mean": mean, "n_units": n, "n_active": n_act,
+        "algorithmic_bytes": b_alg, "bytes_moved_by_the_fused_pass": b_moved,
+        "gbs_on_algorithmic_bytes": b_alg / (best * 1e-6) / 1e9, "gbs_on_bytes_moved": b_moved / (best * 1e-6) / 1e9,
+        "frac_of_measured_copy_peak": {"on_algorithmic_bytes": b_alg / (best * 1e-6) / 1e9 / peak,
+                                       "on_bytes_moved": b_moved / (best * 1e-6) / 1e9 / peak},
+        "launches_per_step": {"lump": 2, "v_first": 3},
+        "kernel_break_out": "per-kernel durations of these same launches: profiles/vmajor_selective_step_temporal.md (ncu)",
+        "api": "cocodiff_selective_prologue"}
+    gr = time_graph(torch, lambda: selective(1, binding.LUMP), sq, iters, flush=flush)
+    if gr is not None:
+        out["steps_1_to_7_selective"]["us_step_1_lump_cuda_graph"] = 1e3 * statistics.median(gr)
+    # the paper's own granularity on the same data: per-token units (T = 1), step 1
+    for groups in (1, P):
+        t1 = 1e3 * statistics.median(time_steps(torch, lambda: selective(1, binding.LUMP, 1, groups), sq, iters, 3, flush=flush))
+        n_act1 = int(na.item())
+        b1 = 2 * E * 2 + 12 * n_act1 * H * D * 2
+        out[f"step_1_per_token_units_groups{groups}"] = {
+            "us_cold_l2": t1, "n_units": S, "n_active": n_act1, "algorithmic_bytes": b1,
+            "gbs_on_algorithmic_bytes": b1 / (t1 * 1e-6) / 1e9, "ratio_to_64_token_tiles": t1 / per_step[0]["us_lump"],
+            "launches_per_step": 3}
     return out
 
 
 def next_rows(torch, binding, args):
     """Rows beyond the headline path, on the temporal workload (P=24, S=9216, H=24, D=128):
-    inverse exchange, the two TAPA phases, per-token selection units, and the paper's
-    50-step cache schedule (5 warm-up steps, refresh every 10 steps, linear cache ratio)."""
+    inverse exchange, the two TAPA phases, and the paper's 50-step cache schedule (5 warm-up
+    steps, refresh every 10 steps, linear cache ratio)."""
     cfg = synth.config("temporal")
     P, S, H, D = cfg["P"], cfg["S"], cfg["H"], cfg["D"]
     E = S * H * D
@@ -524,14 +638,8 @@ def next_rows(torch, binding, args):
     binding.rope_table_2d(cs, dev(L["pos"], torch), S, D, cfg["theta"])
     new = lambda n=1: torch.empty(n * E, dtype=torch.int16, device="cuda")
     qh, kh, vh = new(), new(), new()
-    scratch = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
-    sink = torch.zeros(1, dtype=torch.int64, device="cuda")
     sq, sv = torch.cuda.Stream(), torch.cuda.Stream()
-
-    def flush():
-        with torch.cuda.stream(sq):
-            scratch.zero_()
-            torch.sum(scratch.view(torch.int64), dim=0, keepdim=True, out=sink)
+    flush = Flusher(torch, sq)
 
     iters = max(10, min(args.steps, 30))
     out = {}
@@ -550,31 +658,7 @@ def next_rows(torch, binding, args):
     timed("tapa_phase2", lambda: binding.tapa_phase2(*p1, *th, P, S, H, D, stream=sq), 6 * E * 2)
     del p1, th
 
-    # per-token selection units (T = 1): 20 % of the tokens changed strongly
     comp = [new() for _ in range(3)]
-    for T, label in ((1, "selective_step_T1"),):
-        n = S // T
-        rng = np.random.default_rng(0)
-        hot = np.sort(rng.choice(n, int(np.ceil(0.2 * n)), replace=False))
-        cur = synth.bf16_bits_to_f32(L["v"]).reshape(n, -1).copy()
-        cur[hot] += 0.5
-        cur_v = dev(synth.f32_to_bf16_bits(cur).reshape(S, H, D), torch)
-        ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
-        ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
-        metric = torch.zeros(n, dtype=torch.int64, device="cuda")
-        mask = torch.zeros(n, dtype=torch.uint8, device="cuda")
-        idx = torch.zeros(n, dtype=torch.int32, device="cuda")
-        na = torch.zeros(1, dtype=torch.int32, device="cuda")
-        for groups in (1, P):
-            def step():
-                binding.selective_prologue(v, q, k, cur_v, wq, wk, cfg["eps"], cs, P, S, H, D, T, 0.8, groups, metric,
-                                           mask, idx, na, comp[0], comp[1], comp[2], qh, kh, vh, ws, ws_bytes,
-                                           order=binding.LUMP, stream_qk=sq, stream_v=sq)
-            t = statistics.median(time_steps(torch, step, sq, iters, 3, flush=flush))
-            n_act = int(na.item())
-            nbytes = 2 * E * 2 + 12 * n_act * T * H * D * 2
-            out[f"{label}_groups{groups}"] = {"us_cold_l2": 1e3 * t, "n_units": n, "n_active": n_act, "bytes": nbytes,
-                                              "gbs": nbytes / (t * 1e-3) / 1e9}
 
     # the 50-step schedule on 64-token tiles, inputs fixed (timing only), back to back
     T, total, warmup, interval = cfg["T"], 50, 5, 10
@@ -616,7 +700,8 @@ def main():
     ap.add_argument("--only-main", action="store_true",
                     help="run only the headline loop (short launch list for profiling)")
     ap.add_argument("--only-temporal", action="store_true",
-                    help="run only the temporal workload (full step and selective step), for profiling")
+                    help="run only the temporal workload (its eight steps, then the rows beyond the headline path), for profiling")
+    ap.add_argument("--no-next-rows", action="store_true", help="with --only-temporal: the eight steps only")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -624,8 +709,9 @@ def main():
         import torch
         from paper_2604_14561_b200 import binding
         torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-        pc = other_configs(torch, binding, args, names=("temporal",))
-        pc["next_rows_temporal"] = next_rows(torch, binding, args)
+        pc = {"temporal_steps": temporal_rows(torch, binding, args)}
+        if not args.no_next_rows:
+            pc["next_rows_temporal"] = next_rows(torch, binding, args)
         print(json.dumps({"per_config": pc}, ensure_ascii=False))
     else:
         run_ours(args)

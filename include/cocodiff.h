@@ -6,16 +6,21 @@
  * the all-to-all is a device-local permutation.
  *
  * Conventions for every entry point
- *   - Returns 0 (COCODIFF_OK) or a negative cocodiff_status.  On an error
- *     nothing has been enqueued.
+ *   - Returns 0 (COCODIFF_OK) or a negative cocodiff_status.  Arguments are
+ *     checked before anything is enqueued: after every status except
+ *     COCODIFF_CUDA_ERROR nothing has been enqueued.  COCODIFF_CUDA_ERROR means
+ *     the runtime refused a launch or a copy; work that the same call enqueued
+ *     before that stays enqueued, and a call that uses two streams still
+ *     orders stream_qk behind stream_v before it returns.
  *   - Unless a parameter says "host", every pointer is a DEVICE pointer owned
  *     by the caller.  The library allocates no device memory, never
  *     synchronises the device and enqueues only on the streams it is given
  *     (void* = cudaStream_t, NULL = the default stream).  Calls return as soon
  *     as the work is enqueued.
  *   - bf16 tensors are passed as uint16_t bit patterns, row-major, last index
- *     fastest, and must be 16-byte aligned.  Head dimension D is one of
- *     32, 64, 128, 256.
+ *     fastest, and must be 16-byte aligned.  Head dimension D is a multiple of
+ *     8 from 8 to 256 (a row is D/8 16-byte vectors, one per lane of a group of
+ *     lanes; powers of two use every lane of the group).
  *   - Layouts:  SEQ  = [P][S/P][H][D] == [S][H][D]  (rank p owns tokens
  *                      [p*S/P, (p+1)*S/P): the sequence-parallel layout)
  *               HEAD = [P][H/P][S][D] == [H][S][D]  (rank p owns heads
@@ -136,9 +141,10 @@ int cocodiff_prologue_host(const uint16_t *q_host, const uint16_t *k_host, const
  *     (capacity S*H*D elements).
  * prev_v is only read: which step it holds is the caller's policy.
  * workspace: cocodiff_vmajor_workspace_bytes() bytes of scratch, 256-byte
- * aligned; contents are undefined on entry and on exit (the call clears what
- * it needs).  It holds the per-unit accumulators and the block ticket of the
- * fused metric + selection kernel.  Concurrent calls need distinct workspaces. */
+ * aligned; contents are undefined on entry and on exit.  Large units are cut
+ * into pieces that are summed by different thread blocks; the workspace holds
+ * one 64-bit sum per piece (each is stored before it is read, so nothing has
+ * to be cleared).  Concurrent calls need distinct workspaces. */
 size_t cocodiff_vmajor_workspace_bytes(int P, int S, int H, int D, int T);
 int cocodiff_vmajor_select_compact(const uint16_t *prev_v, const uint16_t *cur_v,
                                    int P, int S, int H, int D, int T, double r, int n_groups,
@@ -256,10 +262,10 @@ int cocodiff_tapa_phase2(const uint16_t *q_p1, const uint16_t *k_p1, const uint1
  * a serving process whose memory pool is owned by someone else, a hook that runs
  * while the application is in a no-allocation phase, a real-time loop that must
  * not touch the allocator.  Such callers already own their inputs and outputs
- * but have nowhere to get the small scratch area the fused metric + selection
- * kernel needs (per-unit accumulators and a block ticket).  Here that scratch is
+ * but have nowhere to get the small scratch area the metric pass needs (the
+ * 64-bit sums of the pieces that large units are cut into).  Here that scratch is
  * a fixed array inside the library image on the device: COCODIFF_STATIC_MAX_UNITS
- * 64-bit accumulators plus 256 bytes (about 256 KB), present on every GPU that
+ * 64-bit words plus 256 bytes (about 256 KB), present on every GPU that
  * loads the library until the process exits.
  *
  * Arguments and results are exactly those of cocodiff_vmajor_select_compact
@@ -270,10 +276,11 @@ int cocodiff_tapa_phase2(const uint16_t *q_p1, const uint16_t *k_p1, const uint1
  *     that device current) and remembers it.  Make that first call outside any
  *     stream capture.
  *   - Every call on a device shares the one array, which still holds whatever
- *     the previous call left; each call clears the part it is going to use, on
- *     its stream, before its kernel runs.  Two calls whose work overlaps on the
- *     GPU (different streams, no ordering between them) race on the array and
- *     give wrong selections: order them, or use the workspace-taking call.
+ *     the previous call left; nothing in it has to start at zero, because a
+ *     call stores every word it is going to read before it reads it.  Two calls
+ *     whose work overlaps on the GPU (different streams, no ordering between
+ *     them) race on the array and give wrong selections: order them, or use the
+ *     workspace-taking call.
  *   - No cudaMalloc, cudaFree or other allocating routine is called. */
 #define COCODIFF_STATIC_MAX_UNITS 32768
 int cocodiff_vmajor_select_compact_static(const uint16_t *prev_v, const uint16_t *cur_v,

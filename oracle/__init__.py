@@ -16,30 +16,51 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "cocodiff_oracle.c")
 _SO = os.path.join(_HERE, "libcocodiff_oracle.so")
+_SO_OMP = os.path.join(_HERE, "libcocodiff_oracle_omp.so")     # the same source, all host cores
 _lib = None
+_lib_omp = None
 
 
-def build(force: bool = False) -> str:
-    """Compile the oracle with gcc (no FMA contraction, no fast-math)."""
-    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
-        tmp = _SO + f".tmp{os.getpid()}"
-        subprocess.check_call(["gcc", "-O2", "-std=c99", "-ffp-contract=off", "-fno-fast-math",
-                               "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
-        os.replace(tmp, _SO)
-    return _SO
+def build(force: bool = False, openmp: bool = False) -> str:
+    """Compile the oracle with gcc (no FMA contraction, no fast-math).  openmp=True
+    builds the same source with -fopenmp beside it (used by the benchmark only)."""
+    out = _SO_OMP if openmp else _SO
+    if force or not os.path.exists(out) or os.path.getmtime(out) < os.path.getmtime(_SRC):
+        tmp = out + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-ffp-contract=off", "-fno-fast-math"] +
+                              (["-fopenmp"] if openmp else []) + ["-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, out)
+    return out
+
+
+def _declare(handle):
+    handle.oracle_bf16_to_f32.restype = C.c_float
+    handle.oracle_bf16_to_f32.argtypes = [C.c_uint16]
+    handle.oracle_f32_to_bf16.restype = C.c_uint16
+    handle.oracle_f32_to_bf16.argtypes = [C.c_float]
+    handle.oracle_head_shard_elems.restype = C.c_int64
+    handle.oracle_seq_shard_elems.restype = C.c_int64
+    return handle
 
 
 def lib():
     global _lib
     if _lib is None:
-        _lib = C.CDLL(build())
-        _lib.oracle_bf16_to_f32.restype = C.c_float
-        _lib.oracle_bf16_to_f32.argtypes = [C.c_uint16]
-        _lib.oracle_f32_to_bf16.restype = C.c_uint16
-        _lib.oracle_f32_to_bf16.argtypes = [C.c_float]
-        _lib.oracle_head_shard_elems.restype = C.c_int64
-        _lib.oracle_seq_shard_elems.restype = C.c_int64
+        _lib = _declare(C.CDLL(build()))
     return _lib
+
+
+def use_all_cores(on: bool) -> None:
+    """Route the calls of this module to the OpenMP build (True) or back to the
+    single-threaded build (False).  For the benchmark's CPU-baseline leg."""
+    global _lib, _lib_omp
+    if on:
+        if _lib_omp is None:
+            _lib_omp = _declare(C.CDLL(build(openmp=True)))
+        _lib = _lib_omp
+    else:
+        _lib = None
+        lib()
 
 
 def _p(a):

@@ -1,9 +1,13 @@
 /*
  * CPU oracle for the Ulysses attention-prologue path of CoCoDiff.
  *
- * TEST INFRASTRUCTURE ONLY.  Plain, slow, single-threaded C; it shares no code
- * with the CUDA library and the product never calls it.  Only the tests, the
- * smoke check and the benchmark's CPU-baseline leg may load this file.
+ * TEST INFRASTRUCTURE ONLY.  Plain, slow C; it shares no code with the CUDA
+ * library and the product never calls it.  Only the tests, the smoke check and
+ * the benchmark's CPU-baseline leg may load this file.  The normal build is
+ * single-threaded.  The benchmark also builds the same source with -fopenmp to
+ * time it on all host cores: the `omp` pragmas below then spread independent
+ * outer loops (tokens, messages, units) over the threads; without that flag they
+ * are ignored, and they change no arithmetic either way.
  *
  * What is written out here, with the passage of the paper each part follows:
  *   - the sequence-parallel -> head-parallel exchange of Ulysses (Section II-A)
@@ -121,10 +125,10 @@ int oracle_rope_table_2d(float *cs, const int32_t *pos, int S, int D, double the
 /* w == NULL skips the normalisation.                                       */
 int oracle_norm_rope(const uint16_t *x, const uint16_t *w, float eps, const float *cs,
                      int S, int H, int D, uint16_t *y_bf16, float *y_f32) {
-    if (D % 2 != 0) return ORACLE_BAD;
-    float *row = (float *)malloc(sizeof(float) * (size_t)D);
-    if (!row) return ORACLE_BAD;
+    if (D % 2 != 0 || D < 2 || D > 65536) return ORACLE_BAD;
+#pragma omp parallel for schedule(static)
     for (int s = 0; s < S; ++s) {
+        float row[D]; /* one row at a time, private to the token's loop iteration */
         for (int h = 0; h < H; ++h) {
             const size_t base = ((size_t)s * H + h) * D;
             for (int j = 0; j < D; ++j) row[j] = bf16_to_f32(x[base + j]);
@@ -154,7 +158,6 @@ int oracle_norm_rope(const uint16_t *x, const uint16_t *w, float eps, const floa
             }
         }
     }
-    free(row);
     return ORACLE_OK;
 }
 
@@ -175,6 +178,7 @@ int oracle_ulysses_a2a(const uint16_t *seq, uint16_t *head, int P, int S, int H,
     uint16_t *recvbuf = (uint16_t *)malloc(2 * (E ? E : 1));
     if (!sendbuf || !recvbuf) { free(sendbuf); free(recvbuf); return ORACLE_BAD; }
     /* pack: sendbuf[src][dst][s_l][h_l][:] */
+#pragma omp parallel for collapse(2) schedule(static)
     for (int src = 0; src < P; ++src)
         for (int dst = 0; dst < P; ++dst)
             for (int sl = 0; sl < Sl; ++sl)
@@ -184,10 +188,12 @@ int oracle_ulysses_a2a(const uint16_t *seq, uint16_t *head, int P, int S, int H,
                     memcpy(to, from, 2 * (size_t)D);
                 }
     /* the wire: recvbuf[dst][src] = sendbuf[src][dst] */
+#pragma omp parallel for collapse(2) schedule(static)
     for (int src = 0; src < P; ++src)
         for (int dst = 0; dst < P; ++dst)
             memcpy(recvbuf + ((size_t)dst * P + src) * msg, sendbuf + ((size_t)src * P + dst) * msg, 2 * msg);
     /* unpack: HEAD[dst][h_l][src*Sl + s_l][:] */
+#pragma omp parallel for collapse(2) schedule(static)
     for (int dst = 0; dst < P; ++dst)
         for (int src = 0; src < P; ++src)
             for (int sl = 0; sl < Sl; ++sl)
@@ -308,6 +314,7 @@ int oracle_vmajor_metric(const uint16_t *prev_v, const uint16_t *cur_v, int P, i
     if (!shapes_ok(P, S, H, D) || T < 1 || (S / P) % T != 0) return ORACLE_BAD;
     const int n = S / T;
     const size_t unit = (size_t)T * H * D;
+#pragma omp parallel for schedule(static)
     for (int u = 0; u < n; ++u) {
         uint64_t acc = 0;
         for (size_t e = 0; e < unit; ++e) {

@@ -195,7 +195,7 @@ def selective_prologue(prev_v, q, k, v, wq, wk, eps, cs, P, S, H, D, T, r, n_gro
                  _stream(stream_qk), _stream(stream_v), check=check)
 
 
-STATIC_MAX_UNITS = 32768
+STATIC_MAX_UNITS = 32768     # COCODIFF_STATIC_MAX_UNITS of include/cocodiff.h (a test keeps the two equal)
 
 
 def vmajor_select_compact_static(prev_v, cur_v, P, S, H, D, T, r, n_groups, metric, mask, idx, n_active,

@@ -30,9 +30,7 @@ def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False
         return out
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = out + f".tmp{os.getpid()}"
-    extra = os.environ.get("COCODIFF_NVCC_EXTRA", "").split()
-    if debug_bounds:
-        extra.append("-DCOCODIFF_DEBUG_BOUNDS")
+    extra = ["-DCOCODIFF_DEBUG_BOUNDS"] if debug_bounds else []
     cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + \
           ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)

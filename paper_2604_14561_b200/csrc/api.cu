@@ -33,7 +33,8 @@ bool overlap(const void *a, size_t na, const void *b, size_t nb) {
     return x < y + nb && y < x + na;
 }
 
-bool supported_d(int D) { return D == 32 || D == 64 || D == 128 || D == 256; }
+// a row is D/8 16-byte vectors, at most one per lane of a warp
+bool supported_d(int D) { return D >= 8 && D <= 256 && D % 8 == 0; }
 
 int check_shape(int P, int S, int H, int D) {
     if (P < 1 || S < 0 || H < 1) return COCODIFF_INVALID_ARG;
@@ -66,6 +67,12 @@ int get_events(ForkJoin **out) {
         CK(cudaEventCreateWithFlags(&fj.join, cudaEventDisableTiming));
     }
     *out = &fj;
+    return COCODIFF_OK;
+}
+
+int join_streams(ForkJoin *fj, cudaStream_t sq, cudaStream_t sv) {
+    CK(cudaEventRecord(fj->join, sv));
+    CK(cudaStreamWaitEvent(sq, fj->join, 0));
     return COCODIFF_OK;
 }
 
@@ -102,6 +109,7 @@ MoveParams seq_to_head(int S, int H, int D) {
     std::memset(&p, 0, sizeof p);
     p.n_slots = S;
     p.H = H;
+    p.D = D;
     p.src_tok = (long long)H * D;
     p.src_head = D;
     p.dst_tok = D;
@@ -123,11 +131,11 @@ int exchange(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *
     if (order == COCODIFF_LUMP || !two_streams) {
         // one launch; V's blocks come first in the grid
         MoveParams p = base;
-        if (v) p.job[p.njobs++] = MoveJob{v, vh, nullptr};
-        if (q) p.job[p.njobs++] = MoveJob{q, qh, wq};
-        if (k) p.job[p.njobs++] = MoveJob{k, kh, wk};
+        if (v) p.job[p.njobs++] = MoveJob{v, vh, nullptr, nullptr};
+        if (q) p.job[p.njobs++] = MoveJob{q, qh, wq, nullptr};
+        if (k) p.job[p.njobs++] = MoveJob{k, kh, wk, nullptr};
         if (p.njobs == 0) return COCODIFF_OK;
-        CK(launch_move(p, D, sq));
+        CK(launch_move(p, sq));
         return COCODIFF_OK;
     }
     ForkJoin *fj = nullptr;
@@ -136,15 +144,16 @@ int exchange(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *
     CK(cudaEventRecord(fj->fork, sq));
     CK(cudaStreamWaitEvent(sv, fj->fork, 0));
     MoveParams pv = base;
-    pv.job[pv.njobs++] = MoveJob{v, vh, nullptr};
-    CK(launch_move(pv, D, sv));
+    pv.job[pv.njobs++] = MoveJob{v, vh, nullptr, nullptr};
     MoveParams pqk = base;
-    if (q) pqk.job[pqk.njobs++] = MoveJob{q, qh, wq};
-    if (k) pqk.job[pqk.njobs++] = MoveJob{k, kh, wk};
-    CK(launch_move(pqk, D, sq));
-    CK(cudaEventRecord(fj->join, sv));
-    CK(cudaStreamWaitEvent(sq, fj->join, 0));
-    return COCODIFF_OK;
+    if (q) pqk.job[pqk.njobs++] = MoveJob{q, qh, wq, nullptr};
+    if (k) pqk.job[pqk.njobs++] = MoveJob{k, kh, wk, nullptr};
+    cudaError_t e = launch_move(pv, sv);
+    if (e == cudaSuccess) e = launch_move(pqk, sq);
+    // whatever happened, stream_qk is ordered behind stream_v again
+    const int rj = join_streams(fj, sq, sv);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return rj;
 }
 
 int check_pairs(const uint16_t *const in[3], uint16_t *const out[3], size_t bytes) {
@@ -162,9 +171,13 @@ int check_pairs(const uint16_t *const in[3], uint16_t *const out[3], size_t byte
 
 
 // ---- V-Major helpers --------------------------------------------------------
-size_t vmajor_ws_bytes(int S, int T) {
-    const size_t n = (size_t)(S / T);
-    return ((n * 8 + 255) / 256) * 256 + 256;  // accumulators, then the ticket
+// Scratch of the metric pass: one 64-bit sum per piece of a unit (see plan_metric),
+// plus a spare 256 bytes.  Units that are not cut (parts == 1) need no scratch: their
+// sums go straight to the caller's metric array.
+size_t vmajor_ws_bytes(int S, int H, int D, int T) {
+    const long long n = S / T;
+    const MetricPlan pl = plan_metric((int)n, (long long)T * H * D / 8);
+    return (((size_t)n * pl.parts * 8 + 255) / 256) * 256 + 256;
 }
 
 // Token slots that the selection rule leaves active: (n - n_groups * floor(r * g)) * T.
@@ -188,7 +201,7 @@ int check_select(const uint16_t *prev_v, const uint16_t *cur_v, int P, int S, in
         (reinterpret_cast<uintptr_t>(metric) & 7u) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
         (reinterpret_cast<uintptr_t>(n_active) & 3u))
         return COCODIFF_MISALIGNED;
-    if (workspace_bytes < vmajor_ws_bytes(S, T)) return COCODIFF_WORKSPACE_TOO_SMALL;
+    if (workspace_bytes < vmajor_ws_bytes(S, H, D, T)) return COCODIFF_WORKSPACE_TOO_SMALL;
     return COCODIFF_OK;
 }
 
@@ -201,56 +214,74 @@ int check_tiles(const uint16_t *const in[3], uint16_t *const out[3], int S, int 
     return check_pairs(in, out, (size_t)S * H * D * 2);
 }
 
-MetricParams make_metric_params(const uint16_t *prev_v, const uint16_t *cur_v, int S, int H, int D, int T, double r,
-                                int n_groups, uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
-                                void *workspace) {
-    const int n = S / T;
-    const size_t need = vmajor_ws_bytes(S, T);
-    MetricParams mp;
-    std::memset(&mp, 0, sizeof mp);
-    mp.prev = reinterpret_cast<const uint4 *>(prev_v);
-    mp.cur = reinterpret_cast<const uint4 *>(cur_v);
-    mp.acc = reinterpret_cast<unsigned long long *>(workspace);
-    mp.ticket = reinterpret_cast<unsigned int *>(reinterpret_cast<char *>(workspace) + (need - 256));
-    mp.metric = reinterpret_cast<unsigned long long *>(metric);
-    mp.unit_vecs = (long long)T * H * D / 8;
-    mp.chunk_vecs = 128;  // 2 KB of each tensor per warp visit: one group of loads in flight
-    mp.chunks_per_unit = (int)((mp.unit_vecs + mp.chunk_vecs - 1) / mp.chunk_vecs);
-    mp.n_units = n;
-    mp.sel.metric = mp.metric;
-    mp.sel.n = n;
-    mp.sel.n_groups = n_groups;
-    mp.sel.g = n / n_groups;
-    mp.sel.n_cached = (int)std::floor(r * (double)mp.sel.g);
-    mp.sel.mask = mask;
-    mp.sel.idx = idx;
-    mp.sel.n_active = n_active;
-    mp.sel.debug = mp.debug = debug_counter();
-    return mp;
+SelectParams make_select_params(const unsigned long long *metric, int n, double r, int n_groups, uint8_t *mask,
+                                int32_t *idx, int32_t *n_active) {
+    SelectParams sp;
+    std::memset(&sp, 0, sizeof sp);
+    sp.metric = metric;
+    sp.n = n;
+    sp.n_groups = n_groups;
+    sp.g = n / n_groups;
+    sp.n_cached = (int)std::floor(r * (double)sp.g);
+    sp.mask = mask;
+    sp.idx = idx;
+    sp.n_active = n_active;
+    sp.debug = debug_counter();
+    return sp;
 }
 
-int enqueue_metric_select(const uint16_t *prev_v, const uint16_t *cur_v, int S, int H, int D, int T, double r,
-                          int n_groups, uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
-                          void *workspace, cudaStream_t st, int pdl = 0) {
-    MetricParams mp = make_metric_params(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace);
-    mp.pdl = pdl;
-    CK(cudaMemsetAsync(workspace, 0, vmajor_ws_bytes(S, T), st));
-    CK(launch_metric_select(mp, st));
-    return COCODIFF_OK;
+// The metric pass and the selection that follows it.
+struct SelectionPlan {
+    MetricParams mp;
+    SelectParams sp;
+    bool in_consumer;  // few units: every block of the consuming kernel selects for itself
+};
+
+SelectionPlan plan_selection(const uint16_t *prev_v, const uint16_t *cur_v, int S, int H, int D, int T, double r,
+                             int n_groups, uint64_t *metric, uint8_t *mask, int32_t *idx, int32_t *n_active,
+                             void *workspace) {
+    const int n = S / T;
+    SelectionPlan pl;
+    std::memset(&pl.mp, 0, sizeof pl.mp);
+    const MetricPlan cut = plan_metric(n, (long long)T * H * D / 8);
+    pl.mp.prev = reinterpret_cast<const uint4 *>(prev_v);
+    pl.mp.cur = reinterpret_cast<const uint4 *>(cur_v);
+    pl.mp.unit_vecs = (long long)T * H * D / 8;
+    pl.mp.part_vecs = cut.part_vecs;
+    pl.mp.parts = cut.parts;
+    pl.mp.warp_mode = cut.warp_mode;
+    pl.mp.n_units = n;
+    pl.mp.debug = debug_counter();
+    pl.sp = make_select_params(reinterpret_cast<const unsigned long long *>(metric), n, r, n_groups, mask, idx,
+                               n_active);
+    if (cut.parts == 1) {
+        pl.mp.out = reinterpret_cast<unsigned long long *>(metric);  // whole units: the sums are the metric
+    } else {
+        pl.mp.out = reinterpret_cast<unsigned long long *>(workspace);
+        pl.sp.metric = nullptr;
+        pl.sp.partial = pl.mp.out;
+        pl.sp.metric_out = reinterpret_cast<unsigned long long *>(metric);
+        pl.sp.parts = cut.parts;
+    }
+    pl.in_consumer = n > 0 && n <= kCountMax;
+    return pl;
 }
 
 // Compaction of up to three tensors in one launch; slot order (Q, K, V), V's blocks first.
-MoveParams make_pack_params(const uint16_t *const in[3], uint16_t *const out[3], const uint16_t *wq,
-                            const uint16_t *wk, float eps, const float *cs, const int32_t *idx,
+// cache[i], when given, also receives the rows (the receiver-side scatter in the same pass).
+MoveParams make_pack_params(const uint16_t *const in[3], uint16_t *const out[3], uint16_t *const cache[3],
+                            const uint16_t *wq, const uint16_t *wk, float eps, const float *cs, const int32_t *idx,
                             const int32_t *n_active, int slots, int S, int H, int D, int T) {
     MoveParams p;
     std::memset(&p, 0, sizeof p);
     p.n_slots = slots;
     p.H = H;
+    p.D = D;
     p.src_tok = (long long)H * D;
     p.src_head = D;
     p.dst_tok = D;
     p.dst_head = COMPACT_STRIDE;
+    p.dst2_head = (long long)S * D;
     p.map = MAP_GATHER;
     p.T = T;
     p.n_units = S / T;
@@ -259,19 +290,38 @@ MoveParams make_pack_params(const uint16_t *const in[3], uint16_t *const out[3],
     p.cs = cs;
     p.eps = eps;
     set_extents(p, (long long)S * H * D, (long long)S * H * D, (long long)S * D);
-    if (in[2]) p.job[p.njobs++] = MoveJob{in[2], out[2], nullptr};
-    if (in[0]) p.job[p.njobs++] = MoveJob{in[0], out[0], wq};
-    if (in[1]) p.job[p.njobs++] = MoveJob{in[1], out[1], wk};
+    p.dst2_extent = (long long)S * H * D;
+    if (in[2]) p.job[p.njobs++] = MoveJob{in[2], out[2], nullptr, cache ? cache[2] : nullptr};
+    if (in[0]) p.job[p.njobs++] = MoveJob{in[0], out[0], wq, cache ? cache[0] : nullptr};
+    if (in[1]) p.job[p.njobs++] = MoveJob{in[1], out[1], wk, cache ? cache[1] : nullptr};
     return p;
 }
 
 int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint16_t *wq, const uint16_t *wk,
                  float eps, const float *cs, const int32_t *idx, const int32_t *n_active, int slots, int S,
-                 int H, int D, int T, cudaStream_t st, int pdl = 0) {
-    MoveParams p = make_pack_params(in, out, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T);
-    p.pdl = pdl;
+                 int H, int D, int T, cudaStream_t st) {
+    MoveParams p = make_pack_params(in, out, nullptr, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T);
     if (p.njobs == 0) return COCODIFF_OK;
-    CK(launch_move(p, D, st));
+    CK(launch_move(p, st));
+    return COCODIFF_OK;
+}
+
+// Metric, selection and the compaction (+ scatter) of the given tensors on one stream,
+// chained with programmatic dependent launches.
+int enqueue_select_and_pack(const SelectionPlan &pl, const uint16_t *const in[3], uint16_t *const out[3],
+                            uint16_t *const cache[3], const uint16_t *wq, const uint16_t *wk, float eps,
+                            const float *cs, int slots, int S, int H, int D, int T, cudaStream_t st) {
+    MoveParams p = make_pack_params(in, out, cache, wq, wk, eps, cs, pl.sp.idx, pl.sp.n_active, slots, S, H, D, T);
+    // the consuming kernel selects for itself when it has few units to rank and at least one block
+    const bool consume = p.njobs > 0 && pl.in_consumer && slots > 0;
+    MetricParams mp = pl.mp;
+    mp.pdl = PDL_TRIGGER;
+    CK(launch_metric(mp, st));
+    if (!consume)  // a selection launch: many units, or nothing follows that could select for itself
+        CK(launch_select(pl.sp, st, pl.mp.n_units > 0 ? (PDL_LAUNCH_ATTR | PDL_WAIT_AT_START | PDL_TRIGGER) : 0));
+    if (p.njobs == 0) return COCODIFF_OK;
+    p.pdl = pl.mp.n_units > 0 ? (PDL_LAUNCH_ATTR | PDL_WAIT_AT_START) : 0;
+    CK(launch_selective_move(p, consume ? &pl.sp : nullptr, st));
     return COCODIFF_OK;
 }
 
@@ -281,6 +331,7 @@ MoveParams make_unpack_params(const uint16_t *const in[3], uint16_t *const out[3
     std::memset(&p, 0, sizeof p);
     p.n_slots = slots;
     p.H = H;
+    p.D = D;
     p.src_tok = D;
     p.src_head = COMPACT_STRIDE;
     p.dst_tok = D;
@@ -292,16 +343,15 @@ MoveParams make_unpack_params(const uint16_t *const in[3], uint16_t *const out[3
     p.n_active = n_active;
     set_extents(p, (long long)S * H * D, (long long)S * H * D, 0);
     for (int i = 2; i >= 0; --i)
-        if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr};
+        if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr, nullptr};
     return p;
 }
 
 int enqueue_unpack(const uint16_t *const in[3], uint16_t *const out[3], const int32_t *idx,
-                   const int32_t *n_active, int slots, int S, int H, int D, int T, cudaStream_t st, int pdl = 0) {
+                   const int32_t *n_active, int slots, int S, int H, int D, int T, cudaStream_t st) {
     MoveParams p = make_unpack_params(in, out, idx, n_active, slots, S, H, D, T);
-    p.pdl = pdl;
     if (p.njobs == 0) return COCODIFF_OK;
-    CK(launch_move(p, D, st));
+    CK(launch_move(p, st));
     return COCODIFF_OK;
 }
 
@@ -352,6 +402,7 @@ int cocodiff_qk_norm_rope(const uint16_t *q, const uint16_t *k, uint16_t *q_out,
     std::memset(&p, 0, sizeof p);
     p.n_slots = S;
     p.H = H;
+    p.D = D;
     p.src_tok = p.dst_tok = (long long)H * D;
     p.src_head = p.dst_head = D;
     p.map = MAP_FULL;
@@ -362,7 +413,7 @@ int cocodiff_qk_norm_rope(const uint16_t *q, const uint16_t *k, uint16_t *q_out,
     if (q) p.job[p.njobs++] = MoveJob{q, q_out, wq};
     if (k) p.job[p.njobs++] = MoveJob{k, k_out, wk};
     if (p.njobs == 0) return COCODIFF_OK;
-    CK(launch_move(p, D, (cudaStream_t)stream));
+    CK(launch_move(p, (cudaStream_t)stream));
     return COCODIFF_OK;
 }
 
@@ -393,6 +444,7 @@ int cocodiff_ulysses_a2a_inverse(const uint16_t *q_head, const uint16_t *k_head,
     std::memset(&p, 0, sizeof p);
     p.n_slots = S;
     p.H = H;
+    p.D = D;
     p.src_tok = D;
     p.src_head = (long long)S * D;
     p.dst_tok = (long long)H * D;
@@ -403,7 +455,7 @@ int cocodiff_ulysses_a2a_inverse(const uint16_t *q_head, const uint16_t *k_head,
     for (int i = 2; i >= 0; --i)
         if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr};
     if (p.njobs == 0) return COCODIFF_OK;
-    CK(launch_move(p, D, (cudaStream_t)stream));
+    CK(launch_move(p, (cudaStream_t)stream));
     return COCODIFF_OK;
 }
 
@@ -460,36 +512,45 @@ int cocodiff_prologue_host(const uint16_t *q_host, const uint16_t *k_host, const
     int chunk = (S + n_chunks - 1) / n_chunks;
     chunk = (chunk + 31) / 32 * 32;
     const size_t tok_in = (size_t)H * D, pitch = (size_t)S * D * 2;
-    for (int c = 0, s0 = 0; s0 < S; ++c, s0 += chunk) {
-        const int len = s0 + chunk <= S ? chunk : S - s0;
-        cudaStream_t st = (c % 2 == 0) ? sv : sq;
-        MoveParams p = seq_to_head(S, H, D);
-        p.n_slots = len;
-        p.cs = cs + (size_t)s0 * D;
-        p.eps = eps;
-        set_extents(p, (long long)len * H * D, (long long)E - (long long)s0 * D, (long long)(S - s0) * D);
-        for (int i = 0; i < 3; ++i) {
-            CK(cudaMemcpyAsync(din[i] + s0 * tok_in, hin[i] + s0 * tok_in, (size_t)len * tok_in * 2,
-                               cudaMemcpyHostToDevice, st));
-            p.job[p.njobs++] = MoveJob{din[i] + s0 * tok_in, dout[i] + (size_t)s0 * D, w[i]};
+    auto run_chunks = [&]() -> cudaError_t {
+        cudaError_t e = cudaSuccess;
+        for (int c = 0, s0 = 0; s0 < S; ++c, s0 += chunk) {
+            const int len = s0 + chunk <= S ? chunk : S - s0;
+            cudaStream_t st = (c % 2 == 0) ? sv : sq;
+            MoveParams p = seq_to_head(S, H, D);
+            p.n_slots = len;
+            p.cs = cs + (size_t)s0 * D;
+            p.eps = eps;
+            set_extents(p, (long long)len * H * D, (long long)E - (long long)s0 * D, (long long)(S - s0) * D);
+            for (int i = 0; i < 3; ++i) {
+                e = cudaMemcpyAsync(din[i] + s0 * tok_in, hin[i] + s0 * tok_in, (size_t)len * tok_in * 2,
+                                    cudaMemcpyHostToDevice, st);
+                if (e != cudaSuccess) return e;
+                p.job[p.njobs++] = MoveJob{din[i] + s0 * tok_in, dout[i] + (size_t)s0 * D, w[i], nullptr};
+            }
+            e = launch_move(p, st);
+            if (e != cudaSuccess) return e;
+            for (int i = 0; i < 3; ++i) {
+                e = cudaMemcpy2DAsync(hout[i] + (size_t)s0 * D, pitch, dout[i] + (size_t)s0 * D, pitch,
+                                      (size_t)len * D * 2, (size_t)H, cudaMemcpyDeviceToHost, st);
+                if (e != cudaSuccess) return e;
+            }
         }
-        CK(launch_move(p, D, st));
-        for (int i = 0; i < 3; ++i)
-            CK(cudaMemcpy2DAsync(hout[i] + (size_t)s0 * D, pitch, dout[i] + (size_t)s0 * D, pitch,
-                                 (size_t)len * D * 2, (size_t)H, cudaMemcpyDeviceToHost, st));
-    }
+        return e;
+    };
+    const cudaError_t e = run_chunks();
+    // whatever happened, stream_qk is ordered behind stream_v again
     if (sv != sq) {
-        CK(cudaEventRecord(fj->join, sv));
-        CK(cudaStreamWaitEvent(sq, fj->join, 0));
+        const int rj = join_streams(fj, sq, sv);
+        if (e == cudaSuccess && rj) return rj;
     }
+    if (e != cudaSuccess) return cuda_fail(e);
     return COCODIFF_OK;
 }
 
 size_t cocodiff_vmajor_workspace_bytes(int P, int S, int H, int D, int T) {
-    (void)H;
-    (void)D;
-    if (P < 1 || T < 1 || S < 0) return 0;
-    return vmajor_ws_bytes(S, T);
+    if (P < 1 || T < 1 || S < 0 || H < 1 || !supported_d(D)) return 0;
+    return vmajor_ws_bytes(S, H, D, T);
 }
 
 int cocodiff_vmajor_select(const uint64_t *metric, int n, double r, int n_groups, uint8_t *mask,
@@ -500,16 +561,8 @@ int cocodiff_vmajor_select(const uint64_t *metric, int n, double r, int n_groups
     if ((reinterpret_cast<uintptr_t>(metric) & 7u) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
         (reinterpret_cast<uintptr_t>(n_active) & 3u))
         return COCODIFF_MISALIGNED;
-    SelectParams sp;
-    sp.metric = reinterpret_cast<const unsigned long long *>(metric);
-    sp.n = n;
-    sp.n_groups = n_groups;
-    sp.g = n / n_groups;
-    sp.n_cached = (int)std::floor(r * (double)sp.g);
-    sp.mask = mask;
-    sp.idx = idx;
-    sp.n_active = n_active;
-    sp.debug = debug_counter();
+    const SelectParams sp = make_select_params(reinterpret_cast<const unsigned long long *>(metric), n, r, n_groups,
+                                               mask, idx, n_active);
     CK(launch_select(sp, (cudaStream_t)stream));
     return COCODIFF_OK;
 }
@@ -521,21 +574,17 @@ int cocodiff_vmajor_select_compact(const uint16_t *prev_v, const uint16_t *cur_v
     int rc = check_select(prev_v, cur_v, P, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace,
                           workspace_bytes);
     if (rc) return rc;
-    const uint16_t *in[3] = {nullptr, nullptr, cur_v};
+    const uint16_t *in[3] = {nullptr, nullptr, v_compact ? cur_v : nullptr};
     uint16_t *out[3] = {nullptr, nullptr, v_compact};
     if (v_compact) {
         rc = check_tiles(in, out, S, H, D, idx, n_active);
         if (rc) return rc;
         if (overlap(prev_v, (size_t)S * H * D * 2, v_compact, (size_t)S * H * D * 2)) return COCODIFF_ALIASING;
     }
-    cudaStream_t st = (cudaStream_t)stream;
-    rc = enqueue_metric_select(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, st,
-                               v_compact ? PDL_TRIGGER : 0);
-    if (rc) return rc;
-    if (v_compact)  // the host knows how many units the rule leaves active: exact grid
-        return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, active_slots(S, T, r, n_groups), S,
-                            H, D, T, st, PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
-    return COCODIFF_OK;
+    const SelectionPlan pl = plan_selection(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace);
+    // the host knows how many units the rule leaves active: exact grid
+    return enqueue_select_and_pack(pl, in, out, nullptr, nullptr, nullptr, 0.f, nullptr, active_slots(S, T, r, n_groups),
+                                   S, H, D, T, (cudaStream_t)stream);
 }
 
 int cocodiff_pack_active(const uint16_t *x, const uint16_t *w, float eps, const float *cs,
@@ -636,44 +685,35 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
     // the host knows how many units will be active: grids are sized exactly
     const int slots = active_slots(S, T, r, n_groups);
     cudaStream_t sq = (cudaStream_t)stream_qk, sv = (cudaStream_t)stream_v;
-    // On one stream the three kernels are chained with programmatic dependent launches:
-    // each successor becomes resident while its predecessor drains and orders itself
-    // with griddepcontrol.wait, which hides its launch latency and ramp-up.
-    int unpack_pdl = 0;
-    if (order == COCODIFF_LUMP || sv == sq) {
-        rc = enqueue_metric_select(prev_v, v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, sq,
-                                   PDL_TRIGGER);
-        if (rc) return rc;
-        rc = enqueue_pack(in, comp, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T, sq,
-                          PDL_LAUNCH_ATTR | PDL_WAIT_AT_START | PDL_TRIGGER);
-        if (rc) return rc;
-        unpack_pdl = PDL_LAUNCH_ATTR | PDL_WAIT_AT_START;
-    } else {
-        // V first: metric, selection and V's compaction on stream_v, chained with dependent
-        // launches; Q and K follow on stream_qk once V's part is done, and the scatter is
-        // chained behind their compaction.
-        ForkJoin *fj = nullptr;
-        rc = get_events(&fj);
-        if (rc) return rc;
-        CK(cudaEventRecord(fj->fork, sq));
-        CK(cudaStreamWaitEvent(sv, fj->fork, 0));
-        rc = enqueue_metric_select(prev_v, v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace, sv,
-                                   PDL_TRIGGER);
-        if (rc) return rc;
-        const uint16_t *in_v[3] = {nullptr, nullptr, v};
-        uint16_t *out_v[3] = {nullptr, nullptr, v_compact};
-        rc = enqueue_pack(in_v, out_v, nullptr, nullptr, 0.f, nullptr, idx, n_active, slots, S, H, D, T, sv,
-                          PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
-        if (rc) return rc;
-        CK(cudaEventRecord(fj->join, sv));
-        CK(cudaStreamWaitEvent(sq, fj->join, 0));
-        const uint16_t *in_qk[3] = {q, k, nullptr};
-        uint16_t *out_qk[3] = {q_compact, k_compact, nullptr};
-        rc = enqueue_pack(in_qk, out_qk, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T, sq, PDL_TRIGGER);
-        if (rc) return rc;
-        unpack_pdl = PDL_LAUNCH_ATTR | PDL_WAIT_AT_START;
-    }
-    if (do_unpack) return enqueue_unpack(comp_in, cache, idx, n_active, slots, S, H, D, T, sq, unpack_pdl);
+    const SelectionPlan pl = plan_selection(prev_v, v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, workspace);
+    uint16_t *const *scatter = do_unpack ? cache : nullptr;
+    // One stream: metric pass, (selection,) one compaction + scatter launch for V, Q and K,
+    // chained with programmatic dependent launches: each successor becomes resident while
+    // its predecessor drains and orders itself with griddepcontrol.wait.
+    if (order == COCODIFF_LUMP || sv == sq)
+        return enqueue_select_and_pack(pl, in, comp, scatter, wq, wk, eps, cs, slots, S, H, D, T, sq);
+    // V first: metric, selection and V's compaction + scatter on stream_v; Q and K follow on
+    // stream_qk once V's part is done and read the list that V's part published.
+    ForkJoin *fj = nullptr;
+    rc = get_events(&fj);
+    if (rc) return rc;
+    CK(cudaEventRecord(fj->fork, sq));
+    CK(cudaStreamWaitEvent(sv, fj->fork, 0));
+    const uint16_t *in_v[3] = {nullptr, nullptr, v};
+    uint16_t *out_v[3] = {nullptr, nullptr, v_compact};
+    uint16_t *cache_v[3] = {nullptr, nullptr, v_cache};
+    rc = enqueue_select_and_pack(pl, in_v, out_v, do_unpack ? cache_v : nullptr, nullptr, nullptr, 0.f, nullptr, slots, S, H,
+                                 D, T, sv);
+    // whatever happened on stream_v, stream_qk is ordered behind it again
+    const int rj = join_streams(fj, sq, sv);
+    if (rc) return rc;
+    if (rj) return rj;
+    const uint16_t *in_qk[3] = {q, k, nullptr};
+    uint16_t *out_qk[3] = {q_compact, k_compact, nullptr};
+    uint16_t *cache_qk[3] = {q_cache, k_cache, nullptr};
+    MoveParams p = make_pack_params(in_qk, out_qk, do_unpack ? cache_qk : nullptr, wq, wk, eps, cs, idx, n_active, slots, S,
+                                    H, D, T);
+    CK(launch_selective_move(p, nullptr, sq));
     return COCODIFF_OK;
 }
 
@@ -743,6 +783,7 @@ int cocodiff_tapa_phase1(const uint16_t *q, const uint16_t *k, const uint16_t *v
         std::memset(&p, 0, sizeof p);
         p.n_slots = S;
         p.H = H;
+        p.D = D;
         p.src_tok = p.dst_tok = (long long)H * D;
         p.src_head = p.dst_head = D;
         p.map = MAP_FULL;
@@ -751,7 +792,7 @@ int cocodiff_tapa_phase1(const uint16_t *q, const uint16_t *k, const uint16_t *v
         for (int i = 2; i >= 0; --i)
             if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i] + (size_t)t * E, nullptr};
         if (p.njobs == 0) return COCODIFF_OK;
-        CK(launch_move(p, D, (cudaStream_t)stream));
+        CK(launch_move(p, (cudaStream_t)stream));
     }
     return COCODIFF_OK;
 }
@@ -779,18 +820,18 @@ int cocodiff_tapa_phase2(const uint16_t *q_p1, const uint16_t *k_p1, const uint1
         if (in[i]) { tp.src[tp.n] = in[i]; tp.dst[tp.n] = out[i]; ++tp.n; }
     tp.S = S;
     tp.H = H;
+    tp.D = D;
     tp.Hl = H / P;
     tp.heads_per_block = 8;
     tp.debug = debug_counter();
-    CK(launch_tapa_phase2(tp, D, (cudaStream_t)stream));
+    CK(launch_tapa_phase2(tp, (cudaStream_t)stream));
     return COCODIFF_OK;
 }
 
 // ---------------------------------------------------------------------------
 // Scratch that lives in the library image, for callers that cannot allocate.
 // One array per GPU that loads the library, held until the process exits.
-#define COCODIFF_STATIC_MAX_UNITS_IMPL 32768
-constexpr size_t kStaticScratchBytes = (size_t)COCODIFF_STATIC_MAX_UNITS_IMPL * 8 + 256;
+constexpr size_t kStaticScratchBytes = (size_t)COCODIFF_STATIC_MAX_UNITS * 8 + 256;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 // In host code `g_static_scratch` is only a handle for the runtime, not a device
@@ -818,29 +859,25 @@ int cocodiff_vmajor_select_compact_static(const uint16_t *prev_v, const uint16_t
                                           uint8_t *mask, int32_t *idx, int32_t *n_active,
                                           uint16_t *v_compact, void *stream) {
     // the unit count is checked against the fixed capacity before anything else is looked at
-    if (T >= 1 && S >= 0 && S / T > COCODIFF_STATIC_MAX_UNITS_IMPL) return COCODIFF_WORKSPACE_TOO_SMALL;
+    if (T >= 1 && S >= 0 && S / T > COCODIFF_STATIC_MAX_UNITS) return COCODIFF_WORKSPACE_TOO_SMALL;
     void *scratch = nullptr;
     int rc = static_scratch_address(&scratch);
     if (rc) return rc;
     rc = check_select(prev_v, cur_v, P, S, H, D, T, r, n_groups, metric, mask, idx, n_active, scratch,
                       kStaticScratchBytes);
     if (rc) return rc;
-    const uint16_t *in[3] = {nullptr, nullptr, cur_v};
+    const uint16_t *in[3] = {nullptr, nullptr, v_compact ? cur_v : nullptr};
     uint16_t *out[3] = {nullptr, nullptr, v_compact};
     if (v_compact) {
         rc = check_tiles(in, out, S, H, D, idx, n_active);
         if (rc) return rc;
         if (overlap(prev_v, (size_t)S * H * D * 2, v_compact, (size_t)S * H * D * 2)) return COCODIFF_ALIASING;
     }
-    cudaStream_t st = (cudaStream_t)stream;
-    // enqueue_metric_select clears the accumulators and the ticket it is about to use
-    rc = enqueue_metric_select(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, scratch, st,
-                               v_compact ? PDL_TRIGGER : 0);
-    if (rc) return rc;
-    if (v_compact)  // the host knows how many units the rule leaves active: exact grid
-        return enqueue_pack(in, out, nullptr, nullptr, 0.f, nullptr, idx, n_active, active_slots(S, T, r, n_groups), S,
-                            H, D, T, st, PDL_LAUNCH_ATTR | PDL_WAIT_AT_START);
-    return COCODIFF_OK;
+    // every piece sum the metric pass needs is stored (not accumulated) before it is read:
+    // nothing in the shared array has to be cleared
+    const SelectionPlan pl = plan_selection(prev_v, cur_v, S, H, D, T, r, n_groups, metric, mask, idx, n_active, scratch);
+    return enqueue_select_and_pack(pl, in, out, nullptr, nullptr, nullptr, 0.f, nullptr, active_slots(S, T, r, n_groups),
+                                   S, H, D, T, (cudaStream_t)stream);
 }
 
 long long cocodiff_debug_bounds_violations(void) {
@@ -865,13 +902,14 @@ long long cocodiff_debug_bounds_selftest(const uint16_t *x, uint16_t *y, int S, 
     std::memset(&p, 0, sizeof p);
     p.n_slots = S;
     p.H = H;
+    p.D = D;
     p.src_tok = p.dst_tok = (long long)H * D;
     p.src_head = p.dst_head = D;
     p.map = MAP_FULL;
     p.T = 1;
     set_extents(p, (long long)(S / 2) * H * D, (long long)(S / 2) * H * D, 0);
     p.job[p.njobs++] = MoveJob{x, y, nullptr};
-    if (launch_move(p, D, (cudaStream_t)stream) != cudaSuccess) return -2;
+    if (launch_move(p, (cudaStream_t)stream) != cudaSuccess) return -2;
     return cocodiff_debug_bounds_violations();
 #else
     (void)x; (void)y; (void)S; (void)H; (void)D; (void)stream;

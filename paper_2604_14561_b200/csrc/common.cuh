@@ -20,7 +20,6 @@ enum TokenMap : int {
 enum PdlFlags : int {
     PDL_WAIT_AT_START = 1,   // the kernel consumes its predecessor's results
     PDL_TRIGGER = 2,         // let the successor start as soon as every block of this grid runs
-    PDL_WAIT_AT_END = 4,     // independent of the predecessor, but must not complete before it
     PDL_LAUNCH_ATTR = 8      // host side: launch with programmatic stream serialization
 };
 
@@ -38,6 +37,8 @@ struct MoveJob {
     const uint16_t *src;
     uint16_t *dst;
     const uint16_t *w;   // RMSNorm weight [D]; nullptr = plain move
+    uint16_t *dst2;      // compaction only: the row is also written to its slot of the cached
+                         // head-parallel tensor [H][S][D] (gather and scatter in one pass); or nullptr
 };
 
 // One launch moves up to three tensors (jobs) of identical geometry.  Strides
@@ -49,8 +50,9 @@ struct MoveParams {
     MoveJob job[3];
     int njobs;
     int n_slots;            // token slots covered by the grid (capacity)
-    int H;
+    int H, D;
     long long src_tok, src_head, dst_tok, dst_head;
+    long long dst2_head;    // head stride of job.dst2 (its token stride is D)
     const float *cs;        // [S][D/2][2] or nullptr
     float eps;
     const int32_t *idx;     // active units (MAP_GATHER / MAP_SCATTER)
@@ -60,14 +62,21 @@ struct MoveParams {
     int map;
     int pdl;                // programmatic dependent launch: see PdlFlags
     int head_split;         // blocks per tile along the heads (>= 1); set by the launcher
-    int order;              // block order; set by the launcher
     long long src_extent, dst_extent;  // elements reachable from job.src / job.dst (bounds-checked build)
+    long long dst2_extent;             // elements reachable from job.dst2
     long long cs_extent;               // floats reachable from cs
     unsigned long long *debug;         // violation counter (bounds-checked build), else nullptr
 };
 
+// Selection over n units in n_groups contiguous groups of g.  The metric of unit
+// e is metric[e] when parts == 0, else the sum of partial[e * parts + k], k < parts
+// (the pieces the metric kernel wrote); in that case the sums are also written
+// to metric_out.
 struct SelectParams {
-    const unsigned long long *metric;  // [n]
+    const unsigned long long *metric;   // [n], parts == 0
+    const unsigned long long *partial;  // [n * parts], parts >= 1
+    unsigned long long *metric_out;     // [n], parts >= 1
+    int parts;
     int n, n_groups, g, n_cached;
     uint8_t *mask;
     int32_t *idx;
@@ -75,16 +84,18 @@ struct SelectParams {
     unsigned long long *debug;
 };
 
+// Metric pass: every unit is cut into `parts` contiguous pieces of part_vecs
+// 16-byte vectors; piece (u, k) is summed by one block (warp_mode == 0) or the
+// whole unit by one warp (warp_mode == 1, parts == 1) and stored, without
+// atomics, to out[u * parts + k].
 struct MetricParams {
     const uint4 *prev, *cur;
-    unsigned long long *acc;      // [n] accumulators in the workspace (zero on entry)
-    unsigned int *ticket;         // block ticket in the workspace (zero on entry)
-    unsigned long long *metric;   // [n] out
+    unsigned long long *out;
     long long unit_vecs;          // 16-byte vectors per selection unit
-    int chunks_per_unit;
-    int chunk_vecs;
+    long long part_vecs;
+    int parts;
     int n_units;
-    SelectParams sel;
+    int warp_mode;
     int pdl;                      // PDL_TRIGGER: dependents may start once every block streams
     unsigned long long *debug;
 };
@@ -95,17 +106,35 @@ struct TapaParams {
     const uint16_t *src[3];
     uint16_t *dst[3];
     int n;                 // tensors
-    int S, H, Hl;          // Hl = H / P heads per rank
+    int S, H, D, Hl;       // Hl = H / P heads per rank
     int heads_per_block;
     unsigned long long *debug;
 };
 
-cudaError_t launch_tapa_phase2(const TapaParams &p, int D, cudaStream_t stream);
-cudaError_t launch_move(const MoveParams &p, int D, cudaStream_t stream);
+// How the metric pass cuts the units (host side; also sizes the workspace).
+struct MetricPlan {
+    int parts;
+    long long part_vecs;
+    int warp_mode;
+};
+MetricPlan plan_metric(int n_units, long long unit_vecs);
+
+// Units up to this count are selected by every block of the consuming kernel
+// itself (no selection launch); it is also the largest group the counting
+// selection kernel takes.
+constexpr int kCountMax = 512;
+
+cudaError_t launch_tapa_phase2(const TapaParams &p, cudaStream_t stream);
+cudaError_t launch_move(const MoveParams &p, cudaStream_t stream);
+// Compaction (and scatter into job.dst2) of the active units.  sel != nullptr:
+// every block first runs the selection over sel->n <= kCountMax units itself
+// and block 0 publishes metric, mask, idx and n_active; sel == nullptr: the list
+// is read from p.idx / p.n_active.
+cudaError_t launch_selective_move(const MoveParams &p, const SelectParams *sel, cudaStream_t stream);
 cudaError_t launch_rope_table(float *cs, const int32_t *pos, int S, int D, double theta, cudaStream_t stream);
 // pdl: PDL_LAUNCH_ATTR | PDL_WAIT_AT_START when the metric was produced by the preceding
 // kernel of the stream; PDL_TRIGGER lets the kernel after the selection start early.
 cudaError_t launch_select(const SelectParams &p, cudaStream_t stream, int pdl = 0);
-cudaError_t launch_metric_select(const MetricParams &p, cudaStream_t stream);
+cudaError_t launch_metric(const MetricParams &p, cudaStream_t stream);
 
 }  // namespace cocodiff

@@ -4,92 +4,140 @@
 // sequence-parallel -> head-parallel exchange of Section II-A, its inverse, the
 // compaction of active units and the receiver-side scatter of Section III-D).
 //
-// A row is D*2 bytes = LPR 16-byte vectors, one per lane of an LPR-lane group,
+// A row is D*2 bytes = D/8 16-byte vectors, one per lane of an LPR-lane group,
 // so both sides are accessed with full 128-bit vectors and every 32-byte
 // sector that is touched is used completely.  A thread keeps its token and
 // walks the H heads: the RoPE angles and the norm weight are loaded once per
 // token and reused for every head.  No shared memory, no block barrier.
+//
+// selective_move_kernel is the same mover for one selective step (Section
+// III-D): when the selection covers at most kCountMax units every block first
+// ranks the units itself from the metric kernel's sums (no selection launch and
+// no one-block stage between the metric pass and the data movement); an active
+// row is then read once and written twice, to the compact send buffer and to its
+// slot of the cached head-parallel tensor.
 #include "move_rows.cuh"
+#include "vmajor.cuh"
 
 namespace cocodiff {
 namespace {
 
 using namespace rows;
 
-// Runs griddepcontrol.wait when the thread leaves the kernel (any return path).
-struct PdlTail {
-    int flags;
-    __device__ __forceinline__ explicit PdlTail(int f) : flags(f) {}
-    __device__ __forceinline__ ~PdlTail() {
-        if (flags & PDL_WAIT_AT_END) asm volatile("griddepcontrol.wait;" ::: "memory");
-    }
-};
-
-// Grid: one block per (job, head range, token tile); THREADS x MINB = threads resident per SM.
-template <int LPR, int KIND, int UN, int UP, int THREADS, int MINB, int HINT>
-__global__ void __launch_bounds__(THREADS, MINB) move_rows_kernel(const __grid_constant__ MoveParams p) {
-    if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (p.pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
-    PdlTail tail(p.pdl);  // PDL_WAIT_AT_END: every exit path waits for the predecessor first
-    move_block<LPR, KIND, UN, UP, THREADS, HINT>(p, blockIdx.x);
-}
-
 // Launch shapes measured on B200 at H = 24, D = 128 (21k tokens): 256 threads,
 // 4 blocks per SM (<= 64 registers), evict-first accesses; heads per block and
 // loads in flight per thread depend on what the launch contains.
-constexpr int kThreads = 256, kMinBlocks = 4, kHint = 0;
+constexpr int kThreads = 256, kMinBlocks = 4;
 
-template <int LPR, int KIND, int UN, int UP, int THREADS, int MINB, int HINT>
-cudaError_t launch_variant(MoveParams p, cudaStream_t stream, int head_split = 1, int order = 1) {
-    constexpr int TOK = THREADS / LPR;
-    const long long tiles = ((long long)p.n_slots + TOK - 1) / TOK;
+// Grid: one block per (head range, job, token tile); THREADS x MINB = threads resident per SM.
+template <int LPR, bool PAD, int KIND, int UN, int UP>
+__global__ void __launch_bounds__(kThreads, kMinBlocks) move_rows_kernel(const __grid_constant__ MoveParams p) {
+    if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
+    int n_valid = p.n_slots;
+    if (p.map != MAP_FULL) {
+        // written by an earlier kernel: a coherent load, ordered after griddepcontrol.wait
+        const long long nv = (long long)__ldcg(p.n_active) * p.T;
+        n_valid = nv < (long long)p.n_slots ? (int)nv : p.n_slots;
+        if (n_valid < 0) n_valid = 0;
+    }
+    move_block<LPR, PAD, KIND, UN, UP, kThreads, false>(p, blockIdx.x, p.idx, n_valid);
+}
+
+template <int LPR, bool PAD>
+__global__ void __launch_bounds__(kThreads, kMinBlocks)
+selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constant__ SelectParams sel, const int select_here) {
+    __shared__ vmajor::SmallSel sm;
+    if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int32_t *list = p.idx;
+    long long nv;
+    if (select_here) {
+        nv = (long long)vmajor::select_small<kThreads>(sel, 0, sel.n, sm, blockIdx.x == 0) * p.T;
+        list = sm.idx;
+    } else {
+        nv = (long long)__ldcg(p.n_active) * p.T;
+    }
+    int n_valid = nv < (long long)p.n_slots ? (int)nv : p.n_slots;
+    if (n_valid < 0) n_valid = 0;
+    move_block<LPR, PAD, KIND_MIXED, 4, 4, kThreads, true>(p, blockIdx.x, list, n_valid);
+}
+
+template <typename K, typename... Args>
+cudaError_t launch_grid(K kernel, long long blocks, cudaStream_t stream, int pdl, Args... args) {
+    if (blocks == 0) return cudaSuccess;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (pdl & PDL_LAUNCH_ATTR) ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+long long grid_blocks(MoveParams &p, int lpr, int heads_per_block) {
+    const int tok = kThreads / lpr;
+    const long long tiles = ((long long)p.n_slots + tok - 1) / tok;
+    int head_split = (p.H + heads_per_block - 1) / heads_per_block;
     if (head_split < 1) head_split = 1;
     if (head_split > p.H) head_split = p.H;
     p.head_split = head_split;
-    p.order = order;
-    const long long blocks = tiles * head_split * p.njobs;
-    if (blocks == 0) return cudaSuccess;
-    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    if (p.pdl & PDL_LAUNCH_ATTR) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)blocks);
-        cfg.blockDim = dim3(THREADS);
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, move_rows_kernel<LPR, KIND, UN, UP, THREADS, MINB, HINT>, p);
-    }
-    move_rows_kernel<LPR, KIND, UN, UP, THREADS, MINB, HINT><<<(unsigned)blocks, THREADS, 0, stream>>>(p);
-    return cudaGetLastError();
+    return tiles * head_split * p.njobs;
 }
 
 // Several blocks per token tile shorten the tail of the grid and let V's plain
 // blocks run beside Q/K's arithmetic-heavier ones (head-range-major block order).
-template <int LPR>
-cudaError_t launch_lpr(const MoveParams &p, cudaStream_t stream) {
+template <int LPR, bool PAD>
+cudaError_t launch_lpr(MoveParams p, cudaStream_t stream) {
     int n_norm = 0;
     for (int i = 0; i < p.njobs; ++i) n_norm += p.job[i].w != nullptr;
     if (n_norm == 0)  // 4 heads per block, 4-8 rows in flight per thread
-        return launch_variant<LPR, KIND_PLAIN, 4, 8, kThreads, kMinBlocks, kHint>(p, stream, (p.H + 3) / 4, 1);
+        return launch_grid(move_rows_kernel<LPR, PAD, KIND_PLAIN, 4, 8>, grid_blocks(p, LPR, 4), stream, p.pdl, p);
     if (n_norm == p.njobs)  // 8 heads per block, 4 rows in flight
-        return launch_variant<LPR, KIND_NORM, 4, 8, kThreads, kMinBlocks, kHint>(p, stream, (p.H + 7) / 8, 1);
+        return launch_grid(move_rows_kernel<LPR, PAD, KIND_NORM, 4, 8>, grid_blocks(p, LPR, 8), stream, p.pdl, p);
     // V with Q and/or K in one launch: 12 heads per block, 4 rows in flight on both paths
-    return launch_variant<LPR, KIND_MIXED, 4, 4, kThreads, kMinBlocks, kHint>(p, stream, (p.H + 11) / 12, 1);
+    return launch_grid(move_rows_kernel<LPR, PAD, KIND_MIXED, 4, 4>, grid_blocks(p, LPR, 12), stream, p.pdl, p);
 }
+
+template <int LPR, bool PAD>
+cudaError_t launch_selective_lpr(MoveParams p, const SelectParams *sel, cudaStream_t stream) {
+    static const SelectParams none = {};
+    return launch_grid(selective_move_kernel<LPR, PAD>, grid_blocks(p, LPR, 8), stream, p.pdl, p, sel ? *sel : none,
+                       sel ? 1 : 0);
+}
+
+// D = 8 * lanes; a lane group is padded to the next power of two.
+#define COCODIFF_DISPATCH_D(D, CALL)                                   \
+    switch (((D) % 8 == 0 && (D) >= 8 && (D) <= 256) ? (D) / 8 : 0) {  \
+        case 1: return CALL(1, false);                                 \
+        case 2: return CALL(2, false);                                 \
+        case 3: return CALL(4, true);                                  \
+        case 4: return CALL(4, false);                                 \
+        case 5: case 6: case 7: return CALL(8, true);                  \
+        case 8: return CALL(8, false);                                 \
+        case 9: case 10: case 11: case 12: case 13: case 14: case 15: return CALL(16, true); \
+        case 16: return CALL(16, false);                               \
+        case 32: return CALL(32, false);                               \
+        case 0: return cudaErrorInvalidValue;                          \
+        default: return CALL(32, true);                                \
+    }
 
 }  // namespace
 
-cudaError_t launch_move(const MoveParams &p, int D, cudaStream_t stream) {
-    switch (D) {
-        case 32: return launch_lpr<4>(p, stream);
-        case 64: return launch_lpr<8>(p, stream);
-        case 128: return launch_lpr<16>(p, stream);
-        case 256: return launch_lpr<32>(p, stream);
-        default: return cudaErrorInvalidValue;
-    }
+cudaError_t launch_move(const MoveParams &p, cudaStream_t stream) {
+#define CALL_MOVE(LPR, PAD) launch_lpr<LPR, PAD>(p, stream)
+    COCODIFF_DISPATCH_D(p.D, CALL_MOVE)
+#undef CALL_MOVE
+}
+
+cudaError_t launch_selective_move(const MoveParams &p, const SelectParams *sel, cudaStream_t stream) {
+#define CALL_SEL(LPR, PAD) launch_selective_lpr<LPR, PAD>(p, sel, stream)
+    COCODIFF_DISPATCH_D(p.D, CALL_SEL)
+#undef CALL_SEL
 }
 
 // ---------------------------------------------------------------------------

@@ -1,5 +1,5 @@
 // Device code of the row mover (see move_kernels.cu for the description of the
-// kernel built from it): the per-block work, separate from the launch code.
+// kernels built from it): the per-block work, separate from the launch code.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -45,20 +45,10 @@ __device__ __forceinline__ float group_sum(float v) {
 // (the lump order of issue).  The specialised forms need fewer registers.
 enum JobKind : int { KIND_PLAIN = 0, KIND_NORM = 1, KIND_MIXED = 2 };
 
-// HINT selects the cache policy of the streaming accesses (0: evict-first loads
-// and stores, 1: read-only path loads + evict-first stores, 2: default, 3: loads
-// served by the L2 only).  The policies measured the same on B200; 0 is used.
-template <int HINT>
-__device__ __forceinline__ uint4 ld_row(const uint4 *p) {
-    if (HINT == 0) return __ldcs(p);
-    if (HINT == 1) return __ldg(p);
-    if (HINT == 3) return __ldcg(p);  // L2 only: data written earlier in the same launch by other blocks
-    return *p;
-}
-template <int HINT>
-__device__ __forceinline__ void st_row(uint4 *p, const uint4 v) {
-    if (HINT == 2) *p = v; else __stcs(p, v);
-}
+// Streaming accesses: every row is read once and written once, so both use the
+// evict-first policy (cache policies measured the same on B200).
+__device__ __forceinline__ uint4 ld_row(const uint4 *p) { return __ldcs(p); }
+__device__ __forceinline__ void st_row(uint4 *p, const uint4 v) { __stcs(p, v); }
 
 template <int U>
 struct UnrollTag { static constexpr int value = U; };
@@ -71,40 +61,39 @@ __device__ __forceinline__ void heads_loop(int &h, const int h_hi, F &&body) {
     if constexpr (U > 1) heads_loop<U / 2>(h, h_hi, body);
 }
 
-// One block's share of a move: block id b -> (job, head range, token tile).
-// LPR lanes per row (D = 8 * LPR); KIND: what the launch contains; UN / UP = heads
-// in flight per thread on the norm path / the plain path.  TOK = THREADS / LPR
-// token slots per tile.  Callable from any kernel whose blocks have THREADS threads.
-template <int LPR, int KIND, int UN, int UP, int THREADS, int HINT>
-__device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b) {
-    constexpr int D = LPR * 8;
+// One block's share of a move: block id b -> (head range, job, token tile).
+// A row of D bf16 values is D/8 16-byte vectors, one per lane of an LPR-lane
+// group (LPR a power of two).  PAD = false: D = 8 * LPR; PAD = true: D/8 < LPR and
+// the lanes beyond the row neither load nor store (they add zero to the row's
+// sum of squares).  KIND: what the launch contains; UN / UP = heads in flight per
+// thread on the norm path / the plain path.  TOK = THREADS / LPR token slots per
+// tile.  DUAL: a job may name a second destination (job.dst2), the row's slot
+// in the cached head-parallel tensor, written in the same pass as the compact
+// buffer.  idx_list (shared or global memory) and n_valid (active token slots)
+// are resolved by the calling kernel.
+template <int LPR, bool PAD, int KIND, int UN, int UP, int THREADS, bool DUAL>
+__device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b, const int32_t *idx_list,
+                                           const int n_valid) {
     constexpr int TOK = THREADS / LPR;  // token slots per tile
+    const int D = PAD ? p.D : LPR * 8;
 
-    int n_valid = p.n_slots;
     long long src_head = p.src_head, dst_head = p.dst_head;
-    if (p.map != MAP_FULL) {
-        // written by the preceding kernel: an ordinary (coherent) load, ordered after griddepcontrol.wait
-        const long long nv = (long long)__ldcg(p.n_active) * p.T;
-        n_valid = nv < (long long)p.n_slots ? (int)nv : p.n_slots;
-        if (n_valid < 0) n_valid = 0;
-        if (src_head == COMPACT_STRIDE) src_head = (long long)n_valid * D;
-        if (dst_head == COMPACT_STRIDE) dst_head = (long long)n_valid * D;
-    }
-    // Block id -> (job, head range, token tile).  ORDER 0: job-major (all of V,
-    // then Q, then K); 1: head-range-major (V, Q, K tiles of range 0, then range 1 ...);
-    // 2: tile-major (the jobs and ranges of one tile are neighbours).
+    if (src_head == COMPACT_STRIDE) src_head = (long long)n_valid * D;
+    if (dst_head == COMPACT_STRIDE) dst_head = (long long)n_valid * D;
+    // Block id -> (head range, job, token tile), head-range-major: the V, Q and K
+    // tiles of one head range are neighbours in the grid, so V's plain blocks run
+    // beside the arithmetic-heavier Q/K blocks.
     const unsigned tiles = (unsigned)(p.n_slots + TOK - 1) / TOK;
     const unsigned hsplit = (unsigned)p.head_split, njobs = (unsigned)p.njobs;
-    unsigned tile, y, job_i;
-    {
-        if (p.order == 0) { job_i = b / (tiles * hsplit); const unsigned r = b - job_i * tiles * hsplit; y = r / tiles; tile = r - y * tiles; }
-        else if (p.order == 1) { y = b / (tiles * njobs); const unsigned r = b - y * tiles * njobs; job_i = r / tiles; tile = r - job_i * tiles; }
-        else { tile = b / (njobs * hsplit); const unsigned r = b - tile * njobs * hsplit; job_i = r / hsplit; y = r - job_i * hsplit; }
-    }
+    const unsigned y = b / (tiles * njobs);
+    const unsigned rem = b - y * tiles * njobs;
+    const unsigned job_i = rem / tiles;
+    const unsigned tile = rem - job_i * tiles;
     const int tile0 = (int)tile * TOK;
     if (tile0 >= n_valid) return;  // block-uniform: nothing in this tile
     const long long sh = src_head / 8, dh = dst_head / 8;  // head strides in vectors
     const int lr = (int)threadIdx.x % LPR;
+    const bool lane_on = !PAD || lr < D / 8;
 
     // heads [h_lo, h_hi) of this block
     const int hs = (p.H + (int)hsplit - 1) / (int)hsplit;
@@ -119,14 +108,15 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
     const bool valid = o_raw < n_valid;
     const int o = valid ? o_raw : tile0;
 
-    long long s = o, d = o;
+    long long s = o, d = o, d2 = o;
     if (p.map != MAP_FULL) {
         const int a = o / p.T;
         (void)COCODIFF_IN_BOUNDS(a >= 0 && a < p.n_units, p.debug);
-        int unit = __ldcg(p.idx + a);  // a list that was never written must not send accesses out of bounds
+        int unit = idx_list[a];  // a list that was never written must not send accesses out of bounds
         unit = unit < 0 ? 0 : (unit >= p.n_units ? p.n_units - 1 : unit);
         const long long tk = (long long)unit * p.T + (o - a * p.T);
         if (p.map == MAP_GATHER) s = tk; else d = tk;
+        d2 = tk;
     }
     // bounds-checked build only: is the 16-byte vector at ptr inside its buffer?
     auto src_ok = [&](const uint4 *ptr) {
@@ -137,21 +127,37 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
         return COCODIFF_IN_BOUNDS(reinterpret_cast<const uint16_t *>(ptr) >= job.dst &&
                                   reinterpret_cast<const uint16_t *>(ptr) - job.dst + 8 <= p.dst_extent, p.debug);
     };
+    auto dst2_ok = [&](const uint4 *ptr) {
+        return COCODIFF_IN_BOUNDS(reinterpret_cast<const uint16_t *>(ptr) >= job.dst2 &&
+                                  reinterpret_cast<const uint16_t *>(ptr) - job.dst2 + 8 <= p.dst2_extent, p.debug);
+    };
     (void)src_ok;
     (void)dst_ok;
+    (void)dst2_ok;
     const uint4 *sp = reinterpret_cast<const uint4 *>(job.src + s * p.src_tok) + lr + h_lo * sh;
     uint4 *dp = reinterpret_cast<uint4 *>(job.dst + d * p.dst_tok) + lr + h_lo * dh;
+    // second destination: [H][S][D], token stride D
+    const bool dual = DUAL && job.dst2 != nullptr;
+    const long long dh2 = DUAL ? p.dst2_head / 8 : 0;
+    uint4 *dp2 = DUAL ? reinterpret_cast<uint4 *>(job.dst2 + (dual ? d2 * D : 0)) + lr + h_lo * dh2 : nullptr;
 
     if (KIND == KIND_PLAIN || (KIND == KIND_MIXED && job.w == nullptr)) {
-        if (!valid) return;
+        if (!valid || !lane_on) return;
         int h = h_lo;
         heads_loop<UP>(h, h_hi, [&](auto u_tag) {
             constexpr int U = decltype(u_tag)::value;
             uint4 v[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) { v[u] = src_ok(sp) ? ld_row<HINT>(sp) : make_uint4(0, 0, 0, 0); sp += sh; }
+            for (int u = 0; u < U; ++u) { v[u] = src_ok(sp) ? ld_row(sp) : make_uint4(0, 0, 0, 0); sp += sh; }
 #pragma unroll
-            for (int u = 0; u < U; ++u) { if (dst_ok(dp)) st_row<HINT>(dp, v[u]); dp += dh; }
+            for (int u = 0; u < U; ++u) {
+                if (dst_ok(dp)) st_row(dp, v[u]);
+                dp += dh;
+                if (DUAL) {
+                    if (dual && dst2_ok(dp2)) st_row(dp2, v[u]);
+                    dp2 += dh2;
+                }
+            }
         });
         return;
     }
@@ -164,9 +170,9 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
     float2 ka01, kb01, kc01, kd01, ka23, kb23, kc23, kd23;
     {
         float w[8];
-        unpack8(__ldg(reinterpret_cast<const uint4 *>(job.w) + lr), w);
+        unpack8(lane_on ? __ldg(reinterpret_cast<const uint4 *>(job.w) + lr) : make_uint4(0, 0, 0, 0), w);
         float c[4] = {1.f, 1.f, 1.f, 1.f}, sn[4] = {0.f, 0.f, 0.f, 0.f};
-        if (p.cs != nullptr) {
+        if (p.cs != nullptr && lane_on) {
             // pairs 4*lr .. 4*lr+3 of token s: 8 floats (cos, sin, cos, sin, ...)
             const float4 *tb = reinterpret_cast<const float4 *>(p.cs + s * D) + 2 * lr;
             const bool cs_ok = COCODIFF_IN_BOUNDS(s >= 0 && s * D + 8 * lr + 8 <= p.cs_extent, p.debug);
@@ -212,12 +218,16 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
         constexpr int U = decltype(u_tag)::value;
         uint4 v[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) { v[u] = src_ok(sp) ? ld_row<HINT>(sp) : make_uint4(0, 0, 0, 0); sp += sh; }
+        for (int u = 0; u < U; ++u) { v[u] = (lane_on && src_ok(sp)) ? ld_row(sp) : make_uint4(0, 0, 0, 0); sp += sh; }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const uint4 y = norm_rope_row(v[u]);
-            if (valid && dst_ok(dp)) st_row<HINT>(dp, y);
+            if (valid && lane_on && dst_ok(dp)) st_row(dp, y);
             dp += dh;
+            if (DUAL) {
+                if (dual && valid && lane_on && dst2_ok(dp2)) st_row(dp2, y);
+                dp2 += dh2;
+            }
         }
     });
 }

@@ -19,13 +19,16 @@ namespace {
 constexpr int kThreads = 256;
 
 // One block: TOK = 256 / LPR tokens, heads [blockIdx.y * hpb, ...) of tensor blockIdx.z.
+// A row is D/8 16-byte vectors, one per lane of an LPR-lane group; when D/8 is
+// not a power of two the group is padded and its last lanes stay idle.
 template <int LPR>
 __global__ void __launch_bounds__(kThreads) tapa_phase2_kernel(const __grid_constant__ TapaParams p) {
-    constexpr int D = LPR * 8;
+    const int D = p.D;
     constexpr int TOK = kThreads / LPR;
     const int s = (int)blockIdx.x * TOK + (int)threadIdx.x / LPR;
     if (s >= p.S) return;
     const int lr = (int)threadIdx.x % LPR;
+    if (lr >= D / 8) return;
     const uint16_t *src = blockIdx.z == 0 ? p.src[0] : (blockIdx.z == 1 ? p.src[1] : p.src[2]);
     uint16_t *dst = blockIdx.z == 0 ? p.dst[0] : (blockIdx.z == 1 ? p.dst[1] : p.dst[2]);
     const long long E = (long long)p.S * p.H * D;
@@ -67,14 +70,15 @@ cudaError_t launch_lpr(const TapaParams &p, cudaStream_t stream) {
 
 }  // namespace
 
-cudaError_t launch_tapa_phase2(const TapaParams &p, int D, cudaStream_t stream) {
-    switch (D) {
-        case 32: return launch_lpr<4>(p, stream);
-        case 64: return launch_lpr<8>(p, stream);
-        case 128: return launch_lpr<16>(p, stream);
-        case 256: return launch_lpr<32>(p, stream);
-        default: return cudaErrorInvalidValue;
-    }
+cudaError_t launch_tapa_phase2(const TapaParams &p, cudaStream_t stream) {
+    if (p.D % 8 != 0 || p.D < 8 || p.D > 256) return cudaErrorInvalidValue;
+    const int lanes = p.D / 8;
+    if (lanes <= 1) return launch_lpr<1>(p, stream);
+    if (lanes <= 2) return launch_lpr<2>(p, stream);
+    if (lanes <= 4) return launch_lpr<4>(p, stream);
+    if (lanes <= 8) return launch_lpr<8>(p, stream);
+    if (lanes <= 16) return launch_lpr<16>(p, stream);
+    return launch_lpr<32>(p, stream);
 }
 
 }  // namespace cocodiff

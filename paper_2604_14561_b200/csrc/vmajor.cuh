@@ -7,23 +7,8 @@ namespace cocodiff {
 namespace vmajor {
 
 constexpr int kMetricThreads = 256;
-#ifndef COCODIFF_METRIC_UNROLL
-#define COCODIFF_METRIC_UNROLL 4
-#endif
-#ifndef COCODIFF_METRIC_BLOCKS_PER_SM
-#define COCODIFF_METRIC_BLOCKS_PER_SM 4
-#endif
-constexpr int kMetricUnroll = COCODIFF_METRIC_UNROLL;
-constexpr int kMetricBlocksPerSm = COCODIFF_METRIC_BLOCKS_PER_SM;
-constexpr int kCountMax = 512;  // groups up to this size are ranked by counting
-
-struct SelectSmem {
-    int warp_sums[33];
-    int sel_bin, sel_k;
-    unsigned long long mstar;
-    int t_c;
-    unsigned long long stage[kCountMax];  // small groups: the metrics; also reduction slots
-};
+constexpr int kMetricUnroll = 4;       // 16-byte loads of each tensor in flight per thread
+constexpr int kMetricBlocksPerSm = 4;
 
 // Exclusive prefix sum of v over the block; *total receives the block sum.
 template <int BLOCK>
@@ -72,128 +57,309 @@ __device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v
     return r;
 }
 
-// Threshold form of the rule: with mstar the metric of the unit of rank
-// n_cached-1 in the order (metric, index), unit e is cached iff vals[e] < mstar,
-// or vals[e] == mstar and fewer than t_c units equal to mstar precede it.
-// Every thread owns a contiguous run of units, so two block scans suffice to
-// emit the mask and the ascending list.  vals may live in shared or global memory.
+// The metric of unit e: given directly, or the sum of the pieces the metric
+// kernel stored.  Written by the preceding kernel of the stream: coherent loads.
+__device__ __forceinline__ unsigned long long unit_metric(const SelectParams &p, int e) {
+    if (p.parts == 0) return COCODIFF_IN_BOUNDS(e >= 0 && e < p.n, p.debug) ? __ldcg(p.metric + e) : 0ull;
+    unsigned long long v = 0;
+    for (int k = 0; k < p.parts; ++k)
+        if (COCODIFF_IN_BOUNDS(e >= 0 && e < p.n, p.debug)) v += __ldcg(p.partial + (long long)e * p.parts + k);
+    return v;
+}
+
+// ---------------------------------------------------------------------------
+// Up to kCountMax units, whole groups: every unit is ranked inside its group by
+// counting (metric, index) pairs in shared memory; the units of rank >= n_cached
+// are active.  Leaves the ascending active list in sm.idx and returns its
+// length; with publish the block also writes metric_out, mask, idx and n_active.
+struct SmallSel {
+    unsigned long long m[kCountMax];
+    int idx[kCountMax];
+    unsigned char active[kCountMax];
+    int warp_sums[33];
+};
+
+template <int BLOCK>
+__device__ int select_small(const SelectParams &p, const int base, const int cnt, SmallSel &sm, const bool publish) {
+    const int tid = threadIdx.x;
+    for (int e = tid; e < cnt; e += BLOCK) sm.m[e] = unit_metric(p, base + e);
+    __syncthreads();
+    for (int e = tid; e < cnt; e += BLOCK) {
+        const int g0 = (e / p.g) * p.g;  // base is a multiple of g
+        const unsigned long long my = sm.m[e];
+        int rank = 0;
+        for (int j = g0; j < g0 + p.g; ++j) {
+            const unsigned long long o = sm.m[j];
+            rank += (o < my) | ((o == my) & (j < e));
+        }
+        sm.active[e] = rank >= p.n_cached ? 1 : 0;
+    }
+    __syncthreads();
+    const int per = (cnt + BLOCK - 1) / BLOCK;
+    const int e_lo = tid * per < cnt ? tid * per : cnt;
+    const int e_hi = e_lo + per < cnt ? e_lo + per : cnt;
+    int c = 0;
+    for (int e = e_lo; e < e_hi; ++e) c += sm.active[e];
+    int total;
+    int pos = block_excl_scan<BLOCK>(c, &total, sm.warp_sums);
+    for (int e = e_lo; e < e_hi; ++e)
+        if (sm.active[e]) sm.idx[pos++] = base + e;
+    __syncthreads();
+    if (publish) {
+        const int out_base = (base / p.g) * (p.g - p.n_cached);
+        for (int e = tid; e < cnt; e += BLOCK)
+            if (COCODIFF_IN_BOUNDS(base + e >= 0 && base + e < p.n, p.debug)) {
+                p.mask[base + e] = sm.active[e];
+                if (p.parts != 0) p.metric_out[base + e] = sm.m[e];
+            }
+        for (int a = tid; a < total; a += BLOCK)
+            if (COCODIFF_IN_BOUNDS(out_base + a >= 0 && out_base + a < p.n, p.debug)) p.idx[out_base + a] = sm.idx[a];
+        if (base == 0 && tid == 0) *p.n_active = p.n_groups * (p.g - p.n_cached);
+    }
+    return total;
+}
+
+// ---------------------------------------------------------------------------
+// Large group: one block finds the metric of rank n_cached-1 (mstar) and how
+// many of the units equal to it are cached (t_c), then emits mask and list.
+//
+// Stage 1 (groups of at most 65535 units): a histogram over a 16-bit monotone
+// key of the 64-bit metric - position of the leading one (6 bits) and the ten
+// bits below it - held in shared memory as 65536 16-bit counters.  A scan of the
+// histogram gives the key that contains the wanted rank.  Stage 2 resolves the
+// rank among the units of that key: by counting when they are few, else by
+// 8-bit radix passes over the bits the key does not cover.  Groups beyond 65535
+// units skip stage 1 and run the radix passes over all bits in use.
+constexpr int kLargeBlock = 1024;
+constexpr int kCandMax = 1024;
+
+struct LargeSel {
+    int warp_sums[33];
+    int sel_bin, sel_k;
+    unsigned long long mstar;
+    int t_c;
+    int n_cand;
+    unsigned long long slots[kLargeBlock / 32];
+    unsigned long long cand_val[kCandMax];
+    int cand_idx[kCandMax];
+};
+// dynamic shared memory: 65536 16-bit counters, reused as 32 per-warp 256-bin histograms
+constexpr size_t kLargeDynBytes = 65536 * 2;
+
+__device__ __forceinline__ unsigned key16(unsigned long long v) {
+    if (v < 2) return 0;  // 0 and 1 share the first key
+    const int e = 63 - __clzll((long long)v);
+    const unsigned long long frac = (v << (63 - e)) << 1;  // bits below the leading one, left-aligned
+    return ((unsigned)e << 10) | (unsigned)(frac >> 54);
+}
+// smallest metric with that key
+__device__ __forceinline__ unsigned long long key16_base(unsigned key) {
+    if (key == 0) return 0ull;
+    const int e = (int)(key >> 10);
+    const unsigned long long top = 1024ull | (key & 1023u);  // leading one and ten bits
+    return e >= 10 ? top << (e - 10) : top >> (10 - e);
+}
+// number of low bits of the metric that the key leaves open
+__device__ __forceinline__ int key16_low_bits(unsigned key) {
+    if (key == 0) return 1;
+    const int e = (int)(key >> 10);
+    return e > 10 ? e - 10 : 0;
+}
+
+// 8-bit radix passes from `shift_top` down to 0 over the units with
+// key16 == want_key (want_key < 0: all units); k = wanted rank among them.
+// Leaves the selected low bits in *prefix_out and the rank among equals in *k_out.
+template <int BLOCK>
+__device__ void radix_passes(const unsigned long long *vals, int g, int want_key, int shift_top, int k,
+                             LargeSel &sm, int *warp_hist, unsigned long long *prefix_out, int *k_out) {
+    const int tid = threadIdx.x, warp = tid >> 5;
+    unsigned long long prefix = 0, pmask = 0;
+    int *my_hist = warp_hist + warp * 256;
+    for (int shift = shift_top; shift >= 0; shift -= 8) {
+        for (int i = tid; i < (BLOCK / 32) * 256; i += BLOCK) warp_hist[i] = 0;
+        __syncthreads();
+        for (int e = tid; e < g; e += BLOCK) {
+            const unsigned long long v = vals[e];
+            if ((want_key < 0 || key16(v) == (unsigned)want_key) && (v & pmask) == prefix)
+                atomicAdd(&my_hist[(int)((v >> shift) & 255ull)], 1);
+        }
+        __syncthreads();
+        int c = 0;
+        if (tid < 256)
+            for (int w = 0; w < BLOCK / 32; ++w) c += warp_hist[w * 256 + tid];
+        int total;
+        const int excl = block_excl_scan<BLOCK>(c, &total, sm.warp_sums);
+        if (tid < 256 && c > 0 && excl <= k && k < excl + c) { sm.sel_bin = tid; sm.sel_k = k - excl; }
+        __syncthreads();
+        prefix |= (unsigned long long)sm.sel_bin << shift;
+        pmask |= 0xffull << shift;
+        k = sm.sel_k;
+        __syncthreads();
+    }
+    *prefix_out = prefix;
+    *k_out = k;
+}
+
+// Threshold form of the rule: unit e is cached iff vals[e] < mstar, or
+// vals[e] == mstar and fewer than t_c units equal to mstar precede it.  Every
+// warp owns a contiguous range of units and walks it 32 at a time (coalesced
+// loads, ballots for the running counts), so two block scans suffice to emit
+// the mask and the ascending list.
 template <int BLOCK>
 __device__ void emit_selection(const SelectParams &p, int grp, const unsigned long long *vals, bool none,
                                unsigned long long mstar, int t_c, int *warp_sums) {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int WARPS = BLOCK / 32;
     const int g = p.g, base = grp * g, out_base = grp * (g - p.n_cached);
-    const int per = (g + BLOCK - 1) / BLOCK;
-    const int e_lo = tid * per < g ? tid * per : g;
-    const int e_hi = e_lo + per < g ? e_lo + per : g;
+    const int per_warp = ((g + WARPS - 1) / WARPS + 31) / 32 * 32;
+    const int w_lo = warp * per_warp < g ? warp * per_warp : g;
+    const int w_hi = w_lo + per_warp < g ? w_lo + per_warp : g;
+    const unsigned lt = (1u << lane) - 1u;
+    // ties in this warp's range
     int ties = 0;
     if (!none)
-        for (int e = e_lo; e < e_hi; ++e) ties += vals[e] == mstar;
+        for (int e0 = w_lo; e0 < w_hi; e0 += 32) {
+            const int e = e0 + lane;
+            ties += __popc(__ballot_sync(0xffffffffu, e < w_hi && vals[e] == mstar));
+        }
     int scan_total;
-    int tie_rank = block_excl_scan<BLOCK>(ties, &scan_total, warp_sums);
+    int tie_rank = block_excl_scan<BLOCK>(lane == 0 ? ties : 0, &scan_total, warp_sums);
+    tie_rank = __shfl_sync(0xffffffffu, tie_rank, 0);
+    // active units in this warp's range
     int actives = 0;
     {
         int tr = tie_rank;
-        for (int e = e_lo; e < e_hi; ++e) {
-            const unsigned long long v = vals[e];
-            const bool tie = !none && v == mstar;
-            const bool cached = !none && (v < mstar || (tie && tr < t_c));
-            tr += tie;
-            actives += !cached;
+        for (int e0 = w_lo; e0 < w_hi; e0 += 32) {
+            const int e = e0 + lane;
+            const unsigned long long v = e < w_hi ? vals[e] : 0ull;
+            const bool tie = !none && e < w_hi && v == mstar;
+            const unsigned tb = __ballot_sync(0xffffffffu, tie);
+            const bool cached = !none && e < w_hi && (v < mstar || (tie && tr + __popc(tb & lt) < t_c));
+            actives += __popc(__ballot_sync(0xffffffffu, e < w_hi && !cached));
+            tr += __popc(tb);
         }
     }
-    int pos = block_excl_scan<BLOCK>(actives, &scan_total, warp_sums);
-    for (int e = e_lo; e < e_hi; ++e) {
-        const unsigned long long v = vals[e];
-        const bool tie = !none && v == mstar;
-        const bool cached = !none && (v < mstar || (tie && tie_rank < t_c));
-        tie_rank += tie;
-        if (COCODIFF_IN_BOUNDS(base + e >= 0 && base + e < p.n, p.debug)) p.mask[base + e] = cached ? 0 : 1;
-        if (!cached) {
-            if (COCODIFF_IN_BOUNDS(out_base + pos >= 0 && out_base + pos < p.n, p.debug)) p.idx[out_base + pos] = base + e;
-            ++pos;
+    int pos = block_excl_scan<BLOCK>(lane == 0 ? actives : 0, &scan_total, warp_sums);
+    pos = __shfl_sync(0xffffffffu, pos, 0);
+    for (int e0 = w_lo; e0 < w_hi; e0 += 32) {
+        const int e = e0 + lane;
+        const unsigned long long v = e < w_hi ? vals[e] : 0ull;
+        const bool tie = !none && e < w_hi && v == mstar;
+        const unsigned tb = __ballot_sync(0xffffffffu, tie);
+        const bool cached = !none && e < w_hi && (v < mstar || (tie && tie_rank + __popc(tb & lt) < t_c));
+        const bool active = e < w_hi && !cached;
+        const unsigned ab = __ballot_sync(0xffffffffu, active);
+        if (e < w_hi && COCODIFF_IN_BOUNDS(base + e >= 0 && base + e < p.n, p.debug)) p.mask[base + e] = cached ? 0 : 1;
+        if (active) {
+            const int o = out_base + pos + __popc(ab & lt);
+            if (COCODIFF_IN_BOUNDS(o >= 0 && o < p.n, p.debug)) p.idx[o] = base + e;
         }
+        tie_rank += __popc(tb);
+        pos += __popc(ab);
     }
     if (grp == 0 && tid == 0) *p.n_active = p.n_groups * (g - p.n_cached);
     __syncthreads();
 }
 
-// Small group (g <= kCountMax): every unit is ranked by counting in shared memory.
 template <int BLOCK>
-__device__ void select_group_small(const SelectParams &p, int grp, SelectSmem &sm) {
+__device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm, unsigned *dyn) {
     const int tid = threadIdx.x;
     const int g = p.g, n_cached = p.n_cached;
-    const unsigned long long *m = p.metric + (long long)grp * g;
     const bool none = n_cached == 0;
-    for (int e = tid; e < g; e += BLOCK) sm.stage[e] = m[e];
-    __syncthreads();
-    if (!none) {
-        for (int e = tid; e < g; e += BLOCK) {
-            const unsigned long long my = sm.stage[e];
-            int less = 0, tie_before = 0;
-            for (int j = 0; j < g; ++j) {
-                const unsigned long long o = sm.stage[j];
-                less += o < my;
-                tie_before += (o == my) & (j < e);
-            }
-            if (less + tie_before == n_cached - 1) { sm.mstar = my; sm.t_c = tie_before + 1; }
-        }
-        __syncthreads();
+    // the group's metrics; pieces are summed once and kept in metric_out
+    const unsigned long long *vals;
+    if (p.parts == 0) vals = p.metric + (long long)grp * g;
+    else {
+        for (int e = tid; e < g; e += BLOCK) p.metric_out[(long long)grp * g + e] = unit_metric(p, grp * g + e);
+        __syncthreads();  // this block reads back only what it wrote itself
+        vals = p.metric_out + (long long)grp * g;
     }
-    emit_selection<BLOCK>(p, grp, sm.stage, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm.warp_sums);
-}
-
-// Large group: radix select (8 bits per pass, starting at the highest byte in
-// use) of the metric of rank n_cached-1.  The metrics are staged in dynamic
-// shared memory when they fit (staged != 0); every warp keeps its own histogram
-// so that clustered metrics do not serialise the whole block on one counter.
-template <int BLOCK>
-__device__ void select_group_large(const SelectParams &p, int grp, SelectSmem &sm, unsigned long long *dyn_vals,
-                                   int *warp_hist, int staged) {
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const int g = p.g, n_cached = p.n_cached;
-    const unsigned long long *m = p.metric + (long long)grp * g;
-    const bool none = n_cached == 0;
-    const unsigned long long *vals = m;
-    unsigned long long mx = 0;
-    for (int e = tid; e < g; e += BLOCK) {
-        const unsigned long long v = m[e];
-        if (staged) dyn_vals[e] = v;
-        mx = v > mx ? v : mx;
-    }
-    if (staged) vals = dyn_vals;
-    mx = block_max_u64<BLOCK>(mx, sm.stage);  // also publishes the staged values
     if (!none) {
-        int top = 56;
-        while (top > 0 && (mx >> top) == 0ull) top -= 8;
-        unsigned long long prefix = 0, pmask = 0;
-        int k = n_cached - 1;
-        int *my_hist = warp_hist + warp * 256;
-        for (int shift = top; shift >= 0; shift -= 8) {
-            for (int i = tid; i < (BLOCK / 32) * 256; i += BLOCK) warp_hist[i] = 0;
+        int *warp_hist = reinterpret_cast<int *>(dyn);
+        const int k = n_cached - 1;
+        if (g <= 65535) {
+            // stage 1: 16-bit key histogram, two counters per 32-bit word
+            for (int i = tid; i < 32768; i += BLOCK) dyn[i] = 0;
             __syncthreads();
             for (int e = tid; e < g; e += BLOCK) {
-                const unsigned long long v = vals[e];
-                if ((v & pmask) == prefix) atomicAdd(&my_hist[(int)((v >> shift) & 255ull)], 1);
+                const unsigned key = key16(vals[e]);
+                atomicAdd(&dyn[key >> 1], (key & 1u) ? 0x10000u : 1u);
             }
             __syncthreads();
-            int c = 0;
-            if (tid < 256)
-                for (int w = 0; w < BLOCK / 32; ++w) c += warp_hist[w * 256 + tid];
+            // every thread owns 64 consecutive keys (32 words)
+            unsigned cnt = 0;
+            for (int i = 0; i < 32; ++i) { const unsigned w = dyn[tid * 32 + i]; cnt += (w & 0xffffu) + (w >> 16); }
             int total;
-            const int excl = block_excl_scan<BLOCK>(c, &total, sm.warp_sums);
-            if (tid < 256 && c > 0 && excl <= k && k < excl + c) { sm.sel_bin = tid; sm.sel_k = k - excl; }
+            const int excl = block_excl_scan<BLOCK>((int)cnt, &total, sm.warp_sums);
+            if (cnt > 0 && excl <= k && k < excl + (int)cnt) {
+                int run = excl;
+                for (int i = 0; i < 64; ++i) {
+                    const unsigned w = dyn[tid * 32 + (i >> 1)];
+                    const int c = (int)((i & 1) ? (w >> 16) : (w & 0xffffu));
+                    if (k < run + c) { sm.sel_bin = tid * 64 + i; sm.sel_k = k - run; sm.n_cand = c; break; }
+                    run += c;
+                }
+            }
             __syncthreads();
-            prefix |= (unsigned long long)sm.sel_bin << shift;
-            pmask |= 0xffull << shift;
-            k = sm.sel_k;
+            const unsigned bin = (unsigned)sm.sel_bin;
+            const int kk = sm.sel_k, n_cand = sm.n_cand;
+            const int low_bits = key16_low_bits(bin);
             __syncthreads();
+            if (low_bits == 0) {
+                if (tid == 0) { sm.mstar = key16_base(bin); sm.t_c = kk + 1; }
+            } else if (n_cand <= kCandMax) {
+                // stage 2a: rank the few units of that key by counting
+                if (tid == 0) sm.n_cand = 0;
+                __syncthreads();
+                for (int e = tid; e < g; e += BLOCK) {
+                    const unsigned long long v = vals[e];
+                    if (key16(v) == bin) {
+                        const int slot = atomicAdd(&sm.n_cand, 1);
+                        if (slot < kCandMax) { sm.cand_val[slot] = v; sm.cand_idx[slot] = e; }
+                    }
+                }
+                __syncthreads();
+                for (int i = tid; i < n_cand; i += BLOCK) {
+                    const unsigned long long my = sm.cand_val[i];
+                    const int my_e = sm.cand_idx[i];
+                    int rank = 0, ties_before = 0;
+                    for (int j = 0; j < n_cand; ++j) {
+                        const unsigned long long o = sm.cand_val[j];
+                        const bool tb = (o == my) & (sm.cand_idx[j] < my_e);
+                        rank += (o < my) | tb;
+                        ties_before += tb;
+                    }
+                    if (rank == kk) { sm.mstar = my; sm.t_c = ties_before + 1; }
+                }
+            } else {
+                // stage 2b: radix passes over the bits below the key
+                unsigned long long prefix;
+                int k_eq;
+                radix_passes<BLOCK>(vals, g, (int)bin, 8 * ((low_bits - 1) / 8), kk, sm, warp_hist, &prefix, &k_eq);
+                if (tid == 0) {
+                    const int covered = 8 * ((low_bits - 1) / 8) + 8;
+                    const unsigned long long lowmask = covered >= 64 ? ~0ull : ((1ull << covered) - 1ull);
+                    sm.mstar = (key16_base(bin) & ~lowmask) | prefix;
+                    sm.t_c = k_eq + 1;
+                }
+            }
+        } else {
+            unsigned long long mx = 0;
+            for (int e = tid; e < g; e += BLOCK) { const unsigned long long v = vals[e]; mx = v > mx ? v : mx; }
+            mx = block_max_u64<BLOCK>(mx, sm.slots);
+            int top = 56;
+            while (top > 0 && (mx >> top) == 0ull) top -= 8;
+            unsigned long long prefix;
+            int k_eq;
+            radix_passes<BLOCK>(vals, g, -1, top, k, sm, warp_hist, &prefix, &k_eq);
+            if (tid == 0) { sm.mstar = prefix; sm.t_c = k_eq + 1; }
         }
-        if (tid == 0) { sm.mstar = prefix; sm.t_c = k + 1; }
         __syncthreads();
     }
     emit_selection<BLOCK>(p, grp, vals, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm.warp_sums);
 }
 
+// ---------------------------------------------------------------------------
 // fix(|a - b|): one fp32 subtraction, scale by 2^16, truncate, saturate to 32
 // bits; NaN counts as the saturated value.
 __device__ __forceinline__ unsigned fix16(float a, float b) {
@@ -202,7 +368,7 @@ __device__ __forceinline__ unsigned fix16(float a, float b) {
     return d != d ? 0xffffffffu : r;
 }
 
-__device__ __forceinline__ unsigned long long l1_of_vec(const uint4 a, const uint4 b) {
+__device__ __forceinline__ unsigned long long l1_of_vec_exact(const uint4 a, const uint4 b) {
     const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
     unsigned long long s = 0;
 #pragma unroll
@@ -213,38 +379,53 @@ __device__ __forceinline__ unsigned long long l1_of_vec(const uint4 a, const uin
     return s;
 }
 
-// Streams this block's share of cur_v / prev_v: warp w of n_warps visits chunks
-// w, w + n_warps, ... and adds one 64-bit partial sum per chunk to its unit's
-// accumulator.  chunk ids fit 32 bits (checked by the launcher).
-__device__ __forceinline__ void metric_stream(const MetricParams &p, const unsigned first_warp, const unsigned n_warps) {
-    constexpr int U = kMetricUnroll;
-    const int lane = threadIdx.x & 31;
-    const unsigned total = (unsigned)p.n_units * (unsigned)p.chunks_per_unit;
-    for (unsigned c = first_warp; c < total; c += n_warps) {
-        const unsigned u = c / (unsigned)p.chunks_per_unit;
-        const unsigned k = c - u * (unsigned)p.chunks_per_unit;
-        const long long v0 = (long long)k * p.chunk_vecs;
-        const long long v1 = v0 + p.chunk_vecs < p.unit_vecs ? v0 + p.chunk_vecs : p.unit_vecs;
-        const uint4 *pc = p.cur + (long long)u * p.unit_vecs;
-        const uint4 *pp = p.prev + (long long)u * p.unit_vecs;
-        unsigned long long acc = 0;
-        for (long long v = v0 + lane; v < v1; v += 32 * U) {
-            uint4 a[U], b[U];
+// The same sum without a float-to-integer conversion per element: for
+// |d| * 2^16 < 2^23 the fused multiply-add |d| * 2^16 + 2^23, rounded toward
+// zero, has the truncated value in its mantissa bits (the product is exact and
+// the spacing of floats in [2^23, 2^24) is 1).  A larger difference, Inf or NaN
+// shows as a bit pattern >= that of 2^24; such a vector is redone exactly.
+__device__ __forceinline__ unsigned long long l1_of_vec(const uint4 a, const uint4 b) {
+    const unsigned aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+    unsigned s = 0, top = 0;
 #pragma unroll
-            for (int i = 0; i < U; ++i)
-                if (v + 32 * i < v1) {
-                    const bool ok = COCODIFF_IN_BOUNDS((long long)u * p.unit_vecs + v + 32 * i < (long long)p.n_units * p.unit_vecs, p.debug);
-                    a[i] = ok ? __ldcs(pc + v + 32 * i) : make_uint4(0, 0, 0, 0);
-                    b[i] = ok ? __ldcs(pp + v + 32 * i) : make_uint4(0, 0, 0, 0);
-                }
-#pragma unroll
-            for (int i = 0; i < U; ++i)
-                if (v + 32 * i < v1) acc += l1_of_vec(a[i], b[i]);
-        }
-#pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (lane == 0 && acc != 0 && COCODIFF_IN_BOUNDS(u < (unsigned)p.n_units, p.debug)) atomicAdd(p.acc + u, acc);
+    for (int q = 0; q < 4; ++q) {
+        const float dl = __uint_as_float(aw[q] << 16) - __uint_as_float(bw[q] << 16);
+        const float dh = __uint_as_float(aw[q] & 0xffff0000u) - __uint_as_float(bw[q] & 0xffff0000u);
+        const unsigned ul = __float_as_uint(__fmaf_rz(fabsf(dl), 65536.0f, 8388608.0f));
+        const unsigned uh = __float_as_uint(__fmaf_rz(fabsf(dh), 65536.0f, 8388608.0f));
+        s += ul + uh;
+        top = max(top, max(ul, uh));
     }
+    if (top >= 0x4B800000u) return l1_of_vec_exact(a, b);
+    return (unsigned long long)(s - 8u * 0x4B000000u);  // eight biases of 2^23, modulo 2^32
+}
+
+// Sum over vectors [v0, v1) of one unit, `stride` threads apart starting at
+// v0 + first; U loads of each tensor are in flight per thread.
+__device__ __forceinline__ unsigned long long metric_span(const MetricParams &p, const long long unit_base,
+                                                          const long long v0, const long long v1, const int first,
+                                                          const int stride) {
+    constexpr int U = kMetricUnroll;
+    const uint4 *pc = p.cur + unit_base, *pp = p.prev + unit_base;
+    const long long limit = (long long)p.n_units * p.unit_vecs;
+    (void)limit;
+    unsigned long long acc = 0;
+    for (long long v = v0 + first; v < v1; v += (long long)stride * U) {
+        uint4 a[U], b[U];
+#pragma unroll
+        for (int i = 0; i < U; ++i)
+            if (v + (long long)stride * i < v1) {
+                const bool ok = COCODIFF_IN_BOUNDS(unit_base + v + (long long)stride * i < limit, p.debug);
+                // cur_v is read again by the compaction of the active units: keep it in the L2;
+                // prev_v is not: evict first
+                a[i] = ok ? __ldg(pc + v + (long long)stride * i) : make_uint4(0, 0, 0, 0);
+                b[i] = ok ? __ldcs(pp + v + (long long)stride * i) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+        for (int i = 0; i < U; ++i)
+            if (v + (long long)stride * i < v1) acc += l1_of_vec(a[i], b[i]);
+    }
+    return acc;
 }
 
 }  // namespace vmajor

@@ -4,12 +4,18 @@
 // floor(r*g) units with the smallest (distance, index) are marked cached and the
 // others active; the active indices are emitted ascending.
 //
-// metric kernel: streams both tensors once with 128-bit loads; every warp owns
-// a contiguous chunk of one unit, reduces with shuffles and adds one 64-bit
-// integer per chunk to the unit's accumulator (integer addition: the result
-// does not depend on the order).  The block that takes the last ticket copies
-// the accumulators out and, for small groups, runs the selection in the same
-// launch.  Nothing waits on another block: the ticket is a plain atomic add.
+// metric kernel: streams both tensors once with 128-bit loads.  Large units are
+// cut into contiguous pieces, one block per piece, so that the pieces fill one
+// resident wave; small units (the per-token rule) take one warp each.  Every
+// piece is reduced in registers and shared memory and stored once: no atomics,
+// nothing to clear beforehand, and integer addition makes the result
+// independent of the order.
+//
+// selection: up to kCountMax units are ranked by counting - either by every
+// block of the kernel that consumes the list (see move_kernels.cu) or by
+// vmajor_select_small_kernel; larger groups go to vmajor_select_large_kernel.
+#include <mutex>
+
 #include "vmajor.cuh"
 
 namespace cocodiff {
@@ -18,52 +24,58 @@ namespace {
 using namespace vmajor;
 
 __global__ void __launch_bounds__(256) vmajor_select_small_kernel(const __grid_constant__ SelectParams p, const int pdl) {
-    __shared__ SelectSmem sm;
+    __shared__ SmallSel sm;
     if (pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
-    select_group_small<256>(p, blockIdx.x, sm);
+    select_small<256>(p, (int)blockIdx.x * p.g, p.g, sm, true);  // one group per block
 }
 
-constexpr int kLargeBlock = 1024;
 __global__ void __launch_bounds__(kLargeBlock)
-vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int staged, const int pdl) {
-    __shared__ SelectSmem sm;
+vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int pdl) {
+    __shared__ LargeSel sm;
+    extern __shared__ unsigned dyn_words[];
     if (pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
-    __shared__ int warp_hist[(kLargeBlock / 32) * 256];
-    extern __shared__ unsigned long long dyn_vals[];
-    select_group_large<kLargeBlock>(p, blockIdx.x, sm, dyn_vals, warp_hist, staged);
+    select_group_large<kLargeBlock>(p, blockIdx.x, sm, dyn_words);
 }
 
 __global__ void __launch_bounds__(kMetricThreads, kMetricBlocksPerSm)
-vmajor_metric_kernel(const __grid_constant__ MetricParams p, const int fuse_select) {
-    __shared__ SelectSmem sm;
-    __shared__ int is_last;
-    metric_stream(p, blockIdx.x * (kMetricThreads / 32) + (threadIdx.x >> 5), gridDim.x * (kMetricThreads / 32));
-
-    // This block has streamed its share: a dependent launch may begin to occupy
+vmajor_metric_kernel(const __grid_constant__ MetricParams p) {
+    __shared__ unsigned long long warp_part[kMetricThreads / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned long long acc;
+    if (p.warp_mode) {
+        // one warp per unit, eight consecutive units per block
+        const long long u = (long long)blockIdx.x * (kMetricThreads / 32) + warp;
+        acc = u < p.n_units ? metric_span(p, u * p.unit_vecs, 0, p.unit_vecs, lane, 32) : 0ull;
+    } else {
+        // one block per piece of a unit
+        const long long u = blockIdx.x / (unsigned)p.parts;
+        const long long k = blockIdx.x - u * p.parts;
+        const long long v0 = k * p.part_vecs;
+        const long long v1 = v0 + p.part_vecs < p.unit_vecs ? v0 + p.part_vecs : p.unit_vecs;
+        acc = metric_span(p, u * p.unit_vecs, v0, v1, (int)threadIdx.x, kMetricThreads);
+    }
+    // This thread has issued all its loads: a dependent launch may begin to occupy
     // the SMs (it orders itself behind the whole grid with griddepcontrol.wait).
     if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
-    // The block that draws the last ticket sees every accumulator complete.
-    __threadfence();
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (p.warp_mode) {
+        const long long u = (long long)blockIdx.x * (kMetricThreads / 32) + warp;
+        if (lane == 0 && u < p.n_units) p.out[u] = acc;
+        return;
+    }
+    if (lane == 0) warp_part[warp] = acc;
     __syncthreads();
     if (threadIdx.x == 0) {
-        const unsigned t = atomicAdd(p.ticket, 1u);
-        is_last = (t == gridDim.x - 1) ? 1 : 0;
+        unsigned long long s = 0;
+#pragma unroll
+        for (int w = 0; w < kMetricThreads / 32; ++w) s += warp_part[w];
+        p.out[blockIdx.x] = s;
     }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    for (int u = threadIdx.x; u < p.n_units; u += kMetricThreads) p.metric[u] = __ldcg(p.acc + u);
-    __syncthreads();
-    if (fuse_select)
-        for (int grp = 0; grp < p.sel.n_groups; ++grp) select_group_small<kMetricThreads>(p.sel, grp, sm);
 }
 
-}  // namespace
-
-namespace {
 template <typename... Args>
 cudaError_t launch_maybe_programmatic(void (*kernel)(Args...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                                       int pdl, Args... args) {
@@ -79,48 +91,66 @@ cudaError_t launch_maybe_programmatic(void (*kernel)(Args...), dim3 grid, dim3 b
     cfg.numAttrs = (pdl & PDL_LAUNCH_ATTR) ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
+
 }  // namespace
+
+// Pieces per unit: as many as fill one resident wave of the metric kernel
+// (4 blocks on each of 148 SMs), but no piece under 16 KB of each tensor.
+// Units of at most 16 KB take one warp each.  The plan depends on the shape
+// only, so that it also sizes the workspace.
+MetricPlan plan_metric(int n_units, long long unit_vecs) {
+    MetricPlan pl;
+    pl.parts = 1;
+    pl.part_vecs = unit_vecs;
+    pl.warp_mode = 0;
+    if (n_units <= 0 || unit_vecs <= 0) return pl;
+    constexpr long long kWave = 148 * kMetricBlocksPerSm, kMinPiece = 1024, kWarpUnit = 1024;
+    if (unit_vecs <= kWarpUnit) {
+        pl.warp_mode = 1;
+        return pl;
+    }
+    long long parts = kWave / n_units;
+    const long long most = unit_vecs / kMinPiece;
+    if (parts > most) parts = most;
+    if (parts > 64) parts = 64;
+    if (parts < 1) parts = 1;
+    pl.parts = (int)parts;
+    pl.part_vecs = (unit_vecs + parts - 1) / parts;
+    return pl;
+}
 
 cudaError_t launch_select(const SelectParams &p, cudaStream_t stream, int pdl) {
     if (p.n == 0) return cudaMemsetAsync(p.n_active, 0, sizeof(int32_t), stream);
     if (p.g <= kCountMax)
         return launch_maybe_programmatic(vmajor_select_small_kernel, dim3(p.n_groups), dim3(256), 0, stream, pdl, p, pdl);
-    // stage the group's metrics in shared memory when they fit beside the histograms
-    const size_t want = (size_t)p.g * sizeof(unsigned long long);
-    const size_t limit = 188 * 1024;  // with the 37 KB of static shared memory: inside the 227 KB a block may use
-    const int staged = want <= limit ? 1 : 0;
-    const size_t dyn = staged ? want : 0;
+    // the 128 KB of dynamic shared memory need the opt-in, once per device
+    static std::mutex mu;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        e = cudaFuncSetAttribute(vmajor_select_large_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)limit);
-        if (e != cudaSuccess) return e;
-        attr_set[dev] = true;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!attr_set[dev]) {
+            e = cudaFuncSetAttribute(vmajor_select_large_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kLargeDynBytes);
+            if (e != cudaSuccess) return e;
+            attr_set[dev] = true;
+        }
     }
-    return launch_maybe_programmatic(vmajor_select_large_kernel, dim3(p.n_groups), dim3(kLargeBlock), dyn, stream, pdl,
-                                     p, staged, pdl);
+    return launch_maybe_programmatic(vmajor_select_large_kernel, dim3(p.n_groups), dim3(kLargeBlock), kLargeDynBytes,
+                                     stream, pdl, p, pdl);
 }
 
-cudaError_t launch_metric_select(const MetricParams &p, cudaStream_t stream) {
-    if (p.n_units == 0) return launch_select(p.sel, stream);
-    // One resident wave (4 blocks of 256 threads per SM); its warps walk the chunks.
-    const long long total = (long long)p.n_units * p.chunks_per_unit;
-    if (total > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    long long blocks = (total + (kMetricThreads / 32) - 1) / (kMetricThreads / 32);
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const long long cap = (long long)sms * kMetricBlocksPerSm;
-    if (blocks > cap) blocks = cap;
-    // one small group: its selection rides in the metric kernel's last block; several
-    // groups or a large one go to their own launch, one block per group
-    const int fuse = (p.sel.g <= kCountMax && p.sel.n_groups <= 2) ? 1 : 0;
-    vmajor_metric_kernel<<<(unsigned)blocks, kMetricThreads, 0, stream>>>(p, fuse);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess || fuse) return e;
-    // the separate selection kernel consumes the metric of the kernel just launched
-    return launch_select(p.sel, stream, PDL_LAUNCH_ATTR | PDL_WAIT_AT_START | (p.pdl & PDL_TRIGGER));
+cudaError_t launch_metric(const MetricParams &p, cudaStream_t stream) {
+    if (p.n_units == 0) return cudaSuccess;
+    long long blocks;
+    if (p.warp_mode) blocks = ((long long)p.n_units + kMetricThreads / 32 - 1) / (kMetricThreads / 32);
+    else blocks = (long long)p.n_units * p.parts;
+    if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    vmajor_metric_kernel<<<(unsigned)blocks, kMetricThreads, 0, stream>>>(p);
+    return cudaGetLastError();
 }
 
 }  // namespace cocodiff

@@ -49,7 +49,7 @@ def _addr(i):
 def test_shape_validation():
     q, k, v, qh, kh, vh = (_addr(i) * 64 for i in range(6))
     ok = dict(P=2, S=8, H=4, D=64)
-    for bad, want in ((dict(P=3), -2), (dict(S=7), -2), (dict(H=3), -2), (dict(D=48), -2), (dict(D=8), -2),
+    for bad, want in ((dict(P=3), -2), (dict(S=7), -2), (dict(H=3), -2), (dict(D=44), -2), (dict(D=4), -2), (dict(D=264), -2),
                       (dict(P=8, S=8, H=4), -2), (dict(P=0), -1), (dict(H=0), -1)):
         a = dict(ok, **bad)
         rc = binding.ulysses_a2a(q, k, v, qh, kh, vh, a["P"], a["S"], a["H"], a["D"], check=False)
@@ -95,6 +95,19 @@ def test_vmajor_validation():
     assert binding.pack_active(cur, None, 0.0, None, idx, na, cur, 2, 64, 4, 64, 8, check=False) == -6
     assert binding.unpack(comp, idx, na, comp + 16, 2, 64, 4, 64, 8, check=False) == -6
     assert binding.unpack(comp, None, na, cur, 2, 64, 4, 64, 8, check=False) == -1
+
+
+def test_static_unit_limit_is_the_headers():
+    text = open(os.path.join(ROOT, "include", "cocodiff.h")).read()
+    m = re.search(r"#define\s+COCODIFF_STATIC_MAX_UNITS\s+(\d+)", text)
+    assert m and int(m.group(1)) == binding.STATIC_MAX_UNITS
+
+
+def test_workspace_size_follows_the_cut_of_the_units():
+    # 144 units of 24576 vectors are cut into 4 pieces each; per-token units are not cut
+    assert binding.vmajor_workspace_bytes(24, 9216, 24, 128, 64) == 144 * 4 * 8 + 256
+    assert binding.vmajor_workspace_bytes(24, 9216, 24, 128, 1) == 9216 * 8 + 256
+    assert binding.vmajor_workspace_bytes(24, 9216, 24, 44, 1) == 0      # unsupported head dimension
 
 
 def test_missing_library_fails_loudly(monkeypatch):

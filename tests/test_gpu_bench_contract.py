@@ -33,6 +33,14 @@ def test_bench_line_has_every_contract_key():
     assert r["traffic"] is None or r["traffic"] > 0.5 * r["algorithmic_bytes_per_launch"]
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and "sample" in c
+    assert c["all_cores"]["cores"] == len(os.sched_getaffinity(0)) and c["all_cores"]["value"] > 0
+    par = c["parity_on_sample"]
+    assert par["v_bit_exact"] is True
+    for t in ("q", "k"):
+        assert par[t]["n_beyond_tolerance"] == 0 and par[t]["n"] > 1e6 and sum(par[t]["ulp_hist"].values()) == par[t]["n"]
+    rep = d["repeats"]
+    assert rep["n"] == 5 and rep["steps_each"] * rep["us_per_layer_median"] >= 19e3
+    assert rep["us_per_layer_min"] <= rep["us_per_layer_median"] <= rep["us_per_layer_max"]
     e = d["e2e"]
     assert e["h2d_bytes_per_step"] == e["d2h_bytes_per_step"] == d["config"]["algorithmic_bytes_per_step"] // 2
     assert 0 < e["value"] < d["value"]
@@ -40,4 +48,11 @@ def test_bench_line_has_every_contract_key():
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
     for bad in ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"):
         assert bad not in d["clocks"]["reasons"]
-    assert set(d["per_config"]) >= {"tiny", "sd3", "qwen768", "temporal", "temporal_selective_step"}
+    pc = d["per_config"]
+    assert set(pc) >= {"launch_floor", "tiny", "sd3", "qwen768", "temporal", "temporal_steps", "next_rows_temporal"}
+    ts = pc["temporal_steps"]
+    sel = ts["steps_1_to_7_selective"]
+    assert [row["step"] for row in sel["per_step"]] == list(range(1, 8))
+    assert all(row["n_active"] == 29 for row in sel["per_step"]) and sel["n_units"] == 144
+    assert sel["algorithmic_bytes"] == 250085376
+    assert 0 < pc["launch_floor"]["us"] < pc["tiny"]["lump"]["us_cold_l2"] + 2.0

@@ -81,6 +81,7 @@ def _run_everything(P, S, H, D, T, r, n_groups, seed):
 SHAPES = [  # P, S, H, D, T, r, n_groups
     (2, 256, 4, 64, 16, 0.8, 1), (3, 99, 3, 32, 11, 0.5, 3), (1, 37, 1, 32, 1, 0.3, 1), (4, 1000, 8, 128, 1, 0.7, 4),
     (2, 130, 2, 256, 5, 0.0, 1), (6, 66, 6, 64, 11, 1.0, 2), (12, 1752, 24, 128, 2, 0.9, 1), (2, 2306, 6, 64, 1153, 0.5, 2),
+    (2, 258, 4, 96, 3, 0.6, 2), (4, 2400, 4, 40, 1, 0.8, 1), (2, 4096, 8, 128, 1024, 0.5, 1), (1, 70, 3, 8, 7, 0.5, 1),
 ]
 
 

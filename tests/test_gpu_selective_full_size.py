@@ -1,0 +1,272 @@
+"""The fused entry points at the size and in the launch shapes the benchmark
+times: `selective_prologue` and `layer_step` on the full temporal workload
+(P=24, S=9216, H=24, D=128), 64-token tiles and per-token units, one global
+group and one group per rank, r = 0.8 and 0.3, every order of issue - each call
+repeated back to back on used workspaces - compared with the CPU oracle
+element by element: metric, mask, index list, the three compact buffers and
+the three caches (Section III-D of the paper; timeline of Figure 4(d)).
+
+The data follow the temporal law of the workload: step 1 = step 0 + N(0, 1e-3)
+everywhere + N(0, 0.5) on a fifth of the 64-token tiles, so the units that stay
+cached have non-zero, nearly tied distances."""
+import functools
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+import oracle
+from paper_2604_14561_b200 import binding, synth
+
+from gpu_util import Guarded, dev, rope_table
+from helpers import assert_norm_rope_close, note
+
+
+@functools.lru_cache(maxsize=None)
+def _data():
+    """Steps 0 and 1 of the temporal sequence, the oracle's normed / rotated Q and K of
+    step 1 and its caches after the full step 0 - computed once for the module."""
+    cfg = synth.config("temporal")
+    P, D = cfg["P"], cfg["D"]
+    seq = synth.TemporalSequence(cfg)
+    step0 = seq.current()
+    hot = seq.advance()
+    step1 = seq.current()
+    cs_ref = oracle.rope_table_2d(seq.pos, D, cfg["theta"])
+    old = dict(zip("qkv", oracle.prologue(step0["q"], step0["k"], step0["v"], seq.wq, seq.wk, cfg["eps"], cs_ref, P)))
+    ref, ref_f = {"v": step1["v"]}, {}
+    for x, w in (("q", seq.wq), ("k", seq.wk)):
+        ref[x], ref_f[x] = oracle.norm_rope(step1[x], w, cfg["eps"], cs_ref, want_f32=True)
+    return dict(cfg=cfg, seq=seq, prev_v=step0["v"], cur=step1, hot=hot, old=old, ref=ref, ref_f=ref_f)
+
+
+@functools.lru_cache(maxsize=2)      # consecutive tests share (T, n_groups, r)
+def _expected(T, n_groups, r):
+    d = _data()
+    P = d["cfg"]["P"]
+    m = oracle.vmajor_metric(d["prev_v"], d["cur"]["v"], P, T)
+    mask, idx, na = oracle.vmajor_select(m, n_groups, r)
+    comp = {x: oracle.pack_active(d["ref"][x], idx, P, T) for x in "qkv"}
+    cache = {x: oracle.unpack(comp[x], idx, d["old"][x].copy(), P, T) for x in "qkv"}
+    return dict(metric=m, mask=mask, idx=idx, na=na, comp=comp, cache=cache)
+
+
+class _Device:
+    """Device copies of the inputs and the output buffers, allocated once."""
+    _one = None
+
+    @classmethod
+    def get(cls):
+        if cls._one is None:
+            cls._one = cls()
+        return cls._one
+
+    def __init__(self):
+        d = _data()
+        cfg, seq = d["cfg"], d["seq"]
+        S, H, D = cfg["S"], cfg["H"], cfg["D"]
+        E = S * H * D
+        self.q, self.k, self.v = (dev(d["cur"][x]) for x in "qkv")
+        self.prev_v = dev(d["prev_v"])
+        self.wq, self.wk = dev(seq.wq), dev(seq.wk)
+        self.cs = rope_table(seq.pos, D, cfg["theta"])
+        self.old = {x: dev(d["old"][x]).reshape(-1) for x in "qkv"}
+        self.comp = {x: Guarded(E) for x in "qkv"}
+        self.cache = {x: Guarded(E) for x in "qkv"}
+        self.metric = torch.zeros(S, dtype=torch.int64, device="cuda")
+        self.mask = torch.zeros(S, dtype=torch.uint8, device="cuda")
+        self.idx = torch.zeros(S, dtype=torch.int32, device="cuda")
+        self.na = torch.zeros(1, dtype=torch.int32, device="cuda")
+        self.ws = torch.full((1 << 20,), 0xAB, dtype=torch.uint8, device="cuda")     # dirty on purpose
+        self.sq, self.sv = torch.cuda.Stream(), torch.cuda.Stream()
+
+
+ORDERS = [(binding.LUMP, False), (binding.V_FIRST, True), (binding.V_FIRST, False)]
+
+
+@pytest.mark.parametrize("order,two_streams", ORDERS, ids=["lump", "v_first_two_streams", "v_first_one_stream"])
+@pytest.mark.parametrize("T,n_groups", [(64, 1), (1, 1), (1, 24)], ids=["tiles64", "per_token", "per_token_per_rank"])
+@pytest.mark.parametrize("r", [0.8, 0.3])
+def test_selective_prologue_full_size(order, two_streams, T, n_groups, r):
+    d, g = _data(), _Device.get()
+    cfg = d["cfg"]
+    P, S, H, D = cfg["P"], cfg["S"], cfg["H"], cfg["D"]
+    n = S // T
+    want = _expected(T, n_groups, r)
+    ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
+    assert ws_bytes <= g.ws.numel()
+    for x in "qkv":
+        g.comp[x].t.fill_(0x5A5A)
+        g.cache[x].t.copy_(g.old[x])
+    g.metric.fill_(-1)
+    g.mask.fill_(9)
+    g.idx.fill_(-1)
+    g.na.fill_(-1)
+    sq = g.sq
+    sv = g.sv if two_streams else sq
+    torch.cuda.synchronize()
+    for _ in range(3):      # back to back, on whatever the previous call left in the workspace
+        binding.selective_prologue(g.prev_v, g.q, g.k, g.v, g.wq, g.wk, cfg["eps"], g.cs, P, S, H, D, T, r, n_groups,
+                                   g.metric, g.mask, g.idx, g.na, g.comp["q"].t, g.comp["k"].t, g.comp["v"].t,
+                                   g.cache["q"].t, g.cache["k"].t, g.cache["v"].t, g.ws, ws_bytes,
+                                   order=order, stream_qk=sq, stream_v=sv)
+    sq.synchronize()
+    na = want["na"]
+    assert np.array_equal(g.metric.cpu().numpy().view(np.uint64)[:n], want["metric"])
+    assert int(g.na.item()) == na
+    assert np.array_equal(g.mask.cpu().numpy()[:n], want["mask"])
+    assert np.array_equal(g.idx.cpu().numpy()[:na], want["idx"])
+    if T == 64 and n_groups == 1 and r == 0.8:
+        assert np.array_equal(want["idx"], d["hot"]), "active set = the strongly perturbed tiles"
+    tok = (want["idx"][:, None].astype(np.int64) * T + np.arange(T)[None, :]).reshape(-1)
+    inactive = np.ones(S, bool)
+    inactive[tok] = False
+    for x in "qkv":
+        comp_ref, cache_ref = want["comp"][x], want["cache"][x]
+        got_c = g.comp[x].host()[:comp_ref.size].reshape(comp_ref.shape)
+        got_cache = g.cache[x].host((H, S, D))
+        assert np.all(g.comp[x].host()[comp_ref.size:] == 0x5A5A), "nothing beyond the compact extent is written"
+        assert np.array_equal(got_cache[:, inactive], cache_ref[:, inactive]), f"{x}: cached rows must not move"
+        if x == "v":
+            assert np.array_equal(got_c, comp_ref) and np.array_equal(got_cache, cache_ref)
+        else:
+            f = np.ascontiguousarray(d["ref_f"][x][tok].transpose(1, 0, 2))
+            assert_norm_rope_close(got_c, comp_ref, f, f"{x} compact")
+            assert np.array_equal(got_cache[:, tok], got_c), "compact buffer and cache receive the same bits"
+        g.comp[x].assert_guards(x + " compact")
+        g.cache[x].assert_guards(x + " cache")
+
+
+def test_layer_step_schedule_full_size():
+    """The first 12 steps of the paper's 50-step schedule (5 warm-up steps, refresh every
+    10, linear cache ratio) on the full temporal workload, step by step against the oracle.
+    The order of issue changes from step to step."""
+    cfg = synth.config("temporal")
+    P, S, H, D, T = cfg["P"], cfg["S"], cfg["H"], cfg["D"], cfg["T"]
+    E, n = S * H * D, S // T
+    total, warmup, interval, n_groups, steps = 50, 5, 10, 1, 12
+    seq = synth.TemporalSequence(cfg)
+    cs_ref, cs = oracle.rope_table_2d(seq.pos, D, cfg["theta"]), rope_table(seq.pos, D, cfg["theta"])
+    wq, wk = dev(seq.wq), dev(seq.wk)
+    cache = {x: Guarded(E) for x in "qkv"}
+    comp = {x: Guarded(E) for x in "qkv"}
+    cache_ref = {x: np.zeros((H, S, D), np.uint16) for x in "qkv"}
+    metric = torch.zeros(n, dtype=torch.int64, device="cuda")
+    mask = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    idx = torch.zeros(n, dtype=torch.int32, device="cuda")
+    na = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
+    ws = torch.full((ws_bytes,), 0xCD, dtype=torch.uint8, device="cuda")
+    sq, sv = torch.cuda.Stream(), torch.cuda.Stream()
+    prev_v = None
+    n_selective, worst = 0, 0.0
+    for step in range(steps):
+        if step:
+            seq.advance()
+        cur = seq.current()
+        d = {x: dev(cur[x]) for x in "qkv"}
+        full, r = binding.cache_schedule(step, total, warmup, interval)
+        assert (full, r) == oracle.cache_schedule(step, total, warmup, interval)
+        order, s_v = ORDERS[step % 3][0], (sv if ORDERS[step % 3][1] else sq)
+        torch.cuda.synchronize()
+        _, sent = binding.layer_step(step, total, warmup, interval, dev(prev_v) if prev_v is not None else d["v"],
+                                     d["q"], d["k"], d["v"], wq, wk, cfg["eps"], cs, P, S, H, D, T, n_groups,
+                                     metric, mask, idx, na, comp["q"].t, comp["k"].t, comp["v"].t,
+                                     cache["q"].t, cache["k"].t, cache["v"].t, ws, ws_bytes,
+                                     order=order, stream_qk=sq, stream_v=s_v)
+        sq.synchronize()
+        normed, normed_f = {"v": cur["v"]}, {}
+        for x, w in (("q", seq.wq), ("k", seq.wk)):
+            normed[x], normed_f[x] = oracle.norm_rope(cur[x], w, cfg["eps"], cs_ref, want_f32=True)
+        if full:
+            assert sent == 3 * E
+            tok = np.arange(S)
+            for x in "qkv":
+                cache_ref[x] = oracle.ulysses_a2a(normed[x], P)
+        else:
+            n_selective += 1
+            m_ref = oracle.vmajor_metric(prev_v, cur["v"], P, T)
+            mask_ref, idx_ref, na_ref = oracle.vmajor_select(m_ref, n_groups, r)
+            assert sent == 3 * na_ref * T * H * D
+            assert np.array_equal(metric.cpu().numpy().view(np.uint64), m_ref)
+            assert int(na.item()) == na_ref and np.array_equal(idx.cpu().numpy()[:na_ref], idx_ref)
+            assert np.array_equal(mask.cpu().numpy(), mask_ref)
+            tok = (idx_ref[:, None].astype(np.int64) * T + np.arange(T)[None, :]).reshape(-1)
+            for x in "qkv":
+                oracle.unpack(oracle.pack_active(normed[x], idx_ref, P, T), idx_ref, cache_ref[x], P, T)
+        untouched = np.ones(S, bool)
+        untouched[tok] = False
+        for x in "qkv":
+            got = cache[x].host((H, S, D))
+            assert np.array_equal(got[:, untouched], cache_ref[x][:, untouched]), (x, step)
+            if x == "v":
+                assert np.array_equal(got, cache_ref[x]), step
+            elif len(tok):
+                st = assert_norm_rope_close(got[:, tok], cache_ref[x][:, tok],
+                                            np.ascontiguousarray(normed_f[x][tok].transpose(1, 0, 2)), f"{x} step {step}")
+                worst = max(worst, st["max_err_over_tol"])
+                cache[x].t.copy_(dev(cache_ref[x]).reshape(-1))      # keep both sides bit-aligned
+            cache[x].assert_guards()
+            comp[x].assert_guards()
+        prev_v = cur["v"]
+    assert n_selective >= 5
+    note(f"layer_step, 12 steps at full size: {n_selective} selective steps, worst err/tol {worst:.3f}")
+
+
+def test_cached_v_readings_a_and_b_full_size():
+    """Reading A of "the cached v" (V of the previous step) and reading B (the receivers'
+    copy, refreshed only where units were sent; on the device: the V cache moved back to the
+    sequence-parallel layout) select the same units on the full temporal workload, step by
+    step; what reading B costs is reported as the drift of the V cache from the exact tensor."""
+    cfg = synth.config("temporal")
+    P, S, H, D, T, r, n_groups = cfg["P"], cfg["S"], cfg["H"], cfg["D"], cfg["T"], cfg["r"], cfg["n_groups"]
+    E, n = S * H * D, S // T
+    seq = synth.TemporalSequence(cfg)
+    cs = rope_table(seq.pos, D, cfg["theta"])
+    wq, wk = dev(seq.wq), dev(seq.wk)
+    cur = seq.current()
+    d = {x: dev(cur[x]) for x in "qkv"}
+    cache = {x: Guarded(E) for x in "qkv"}
+    comp = {x: Guarded(E) for x in "qkv"}
+    binding.prologue(d["q"], d["k"], d["v"], cache["q"].t, cache["k"].t, cache["v"].t, wq, wk, cfg["eps"], cs, P, S, H, D)
+    prev_a = d["v"]
+    prev_b = torch.empty(E, dtype=torch.int16, device="cuda")
+    out = {k: (torch.zeros(n, dtype=torch.int64, device="cuda"), torch.zeros(n, dtype=torch.uint8, device="cuda"),
+               torch.zeros(n, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda")) for k in "ab"}
+    ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    ever = np.zeros(n, bool)
+    report = []
+    for step in range(1, 5):
+        hot = seq.advance()
+        cur = seq.current()
+        d = {x: dev(cur[x]) for x in "qkv"}
+        binding.ulysses_a2a_inverse(None, None, cache["v"].t, None, None, prev_b, P, S, H, D)     # the receivers' copy
+        # reading A: selection only; reading B: the whole selective step, which also refreshes the caches
+        binding.vmajor_select_compact(prev_a, d["v"], P, S, H, D, T, r, n_groups, *out["a"], None, ws, ws_bytes)
+        binding.selective_prologue(prev_b, d["q"], d["k"], d["v"], wq, wk, cfg["eps"], cs, P, S, H, D, T, r, n_groups,
+                                   *out["b"], comp["q"].t, comp["k"].t, comp["v"].t,
+                                   cache["q"].t, cache["k"].t, cache["v"].t, ws, ws_bytes, order=binding.LUMP)
+        torch.cuda.synchronize()
+        mask_a, mask_b = out["a"][1].cpu().numpy(), out["b"][1].cpu().numpy()
+        assert np.array_equal(mask_a, mask_b), step
+        assert np.array_equal(np.flatnonzero(mask_b), hot)
+        # oracle on reading A's inputs
+        m_ref = oracle.vmajor_metric(prev_a.cpu().numpy().view(np.uint16).reshape(S, H, D), cur["v"], P, T)
+        assert np.array_equal(out["a"][0].cpu().numpy().view(np.uint64), m_ref)
+        assert np.array_equal(oracle.vmajor_select(m_ref, n_groups, r)[0], mask_a)
+        ever |= mask_b.astype(bool)
+        exact = oracle.ulysses_a2a(cur["v"], P)
+        got = cache["v"].host((H, S, D))
+        stale = (got != exact).any(axis=(0, 2)).reshape(n, T).any(axis=1)
+        assert np.array_equal(stale, ~mask_b.astype(bool)), "exact where a unit was sent in this step, stale elsewhere"
+        delta = np.abs(synth.bf16_bits_to_f32(got).astype(np.float64) - synth.bf16_bits_to_f32(exact))
+        report.append(dict(step=step, stale_units=int(stale.sum()), max_abs_delta=float(delta.max()),
+                           mean_abs_delta_on_stale_rows=float(delta.reshape(H, n, T, D)[:, stale].mean())))
+        for x in "qkv":
+            cache[x].assert_guards()
+        prev_a = d["v"]
+    assert 0 < int(ever.sum()) < n
+    note(f"cached-V readings, full temporal workload: same masks at every step; drift of the V cache {report}")

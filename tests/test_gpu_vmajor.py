@@ -53,7 +53,10 @@ def _pair(S, H, D, T, seed, frac=0.25):
 
 @pytest.mark.parametrize("P,S,H,D,T,n_groups", [
     (2, 256, 4, 64, 16, 1), (2, 256, 4, 64, 16, 2), (4, 512, 4, 128, 1, 4), (4, 512, 4, 128, 1, 1),
-    (3, 96, 3, 32, 8, 12), (1, 40, 2, 256, 5, 1), (8, 2560, 8, 128, 64, 4), (2, 1200, 2, 64, 1, 1)])
+    (3, 96, 3, 32, 8, 12), (1, 40, 2, 256, 5, 1), (8, 2560, 8, 128, 64, 4), (2, 1200, 2, 64, 1, 1),
+    # units cut into pieces (few large units), one block per unit, and head dimensions off the powers of two
+    (2, 1024, 8, 128, 256, 1), (4, 2048, 8, 96, 32, 2), (2, 640, 4, 40, 4, 1), (1, 520, 3, 8, 1, 1),
+    (2, 16384, 2, 64, 8192, 1), (3, 3000, 3, 72, 1, 3)])
 @pytest.mark.parametrize("r", [0.0, 0.3, 0.8, 1.0])
 def test_metric_selection_and_v_compaction(P, S, H, D, T, n_groups, r):
     prev, cur, _ = _pair(S, H, D, T, seed=S + T)
@@ -89,14 +92,23 @@ def test_metric_special_values():
     assert np.all(np.delete(same, 0) == 0)      # NaN - NaN is NaN: unit 0 stays saturated
 
 
-@pytest.mark.parametrize("n,n_groups", [(144, 1), (1000, 1), (1000, 8), (5000, 1), (21024, 1), (4096, 2), (513, 1), (600, 600)])
+@pytest.mark.parametrize("n,n_groups", [(144, 1), (1000, 1), (1000, 8), (5000, 1), (21024, 1), (4096, 2), (513, 1), (600, 600),
+                                        (32768, 1), (30000, 1), (65535, 1), (70000, 1), (140000, 2), (512, 1), (1024, 2)])
 def test_selection_alone_with_ties_and_wide_keys(n, n_groups):
     rng = np.random.default_rng(n + n_groups)
-    for r, kind in ((0.8, "ties"), (0.5, "wide"), (0.999, "ties"), (0.0, "wide"), (1.0, "ties"), (0.25, "equal")):
+    for r, kind in ((0.8, "ties"), (0.5, "wide"), (0.999, "ties"), (0.0, "wide"), (1.0, "ties"), (0.25, "equal"),
+                    (0.8, "sums"), (0.3, "sums"), (0.6, "narrow")):
         if kind == "ties":
             m = rng.integers(0, 7, n).astype(np.uint64)
         elif kind == "equal":
             m = np.full(n, 12345, np.uint64)
+        elif kind == "sums":      # like per-token distances: a tight cluster and a far, wide one
+            m = rng.normal(2.0e5, 3.0e3, n)
+            hot = rng.random(n) < 0.2
+            m[hot] = rng.normal(8.0e7, 2.0e6, int(hot.sum()))
+            m = np.maximum(m, 0).astype(np.uint64)
+        elif kind == "narrow":    # thousands of units inside one key of the coarse histogram
+            m = (np.uint64(3 << 40) + rng.integers(0, 1 << 20, n).astype(np.uint64))
         else:
             m = rng.integers(0, 2 ** 63, n).astype(np.uint64) * np.uint64(2) + rng.integers(0, 2, n).astype(np.uint64)
             m[rng.integers(0, n, n // 4)] = m[0]

@@ -201,3 +201,47 @@ def test_prologue_is_the_composition():
     assert np.array_equal(qh, oracle.norm_rope(L["q"], L["wq"], cfg["eps"], cs).transpose(1, 0, 2))
     assert np.array_equal(kh, oracle.norm_rope(L["k"], L["wk"], cfg["eps"], cs).transpose(1, 0, 2))
     assert not np.array_equal(qh, kh)
+
+
+def test_two_readings_of_the_cached_v_give_the_same_masks():
+    """What "the cached v" of the selection rule holds is not fixed by the paper.
+    Reading A: V of the previous step, refreshed every step (V's Phase 1 is full-size).
+    Reading B: the receivers' copy, refreshed only on the units that were sent.
+    On data that follow the temporal law of the workload (small noise everywhere, a
+    fifth of the tiles strongly perturbed, re-drawn every step) both readings select
+    the same units at every step, and the cache differs from the exact tensor only
+    on units that were never sent, by no more than the accumulated small noise."""
+    cfg = synth.config("temporal")
+    cfg.update(grid=(32, 24), P=4, H=4, D=64, T=16, steps=8)
+    cfg["S"] = 32 * 24
+    P, S, H, D, T, r = cfg["P"], cfg["S"], cfg["H"], cfg["D"], cfg["T"], cfg["r"]
+    n = S // T
+    seq = synth.TemporalSequence(cfg)
+    v0 = seq.current()["v"]
+    prev_a = v0.copy()
+    prev_b = v0.copy()                              # SEQ-layout view of what the receivers hold
+    cache = oracle.ulysses_a2a(v0, P)               # step 0: full exchange
+    ever_sent = np.zeros(n, bool)
+    for step in range(1, cfg["steps"]):
+        hot = seq.advance()
+        v = seq.current()["v"]
+        mask_a, idx_a, _ = oracle.vmajor_select(oracle.vmajor_metric(prev_a, v, P, T), cfg["n_groups"], r)
+        mask_b, idx_b, _ = oracle.vmajor_select(oracle.vmajor_metric(prev_b, v, P, T), cfg["n_groups"], r)
+        assert np.array_equal(mask_a, mask_b), step
+        assert np.array_equal(idx_a, hot)
+        oracle.unpack(oracle.pack_active(v, idx_b, P, T), idx_b, cache, P, T)
+        tok = (idx_b[:, None] * T + np.arange(T)[None, :]).reshape(-1)
+        prev_b[tok] = v[tok]
+        prev_a = v
+        ever_sent[idx_b] = True
+        assert np.array_equal(oracle.ulysses_a2a_inverse(cache, P), prev_b), "reading B is the receivers' copy"
+        exact = oracle.ulysses_a2a(v, P)
+        stale_tok = (cache != exact).any(axis=(0, 2))
+        sent_now = np.zeros(S, bool)
+        sent_now[tok] = True
+        assert not (stale_tok & sent_now).any(), "a unit sent in this step is exact"
+        c64, e64 = synth.bf16_bits_to_f32(cache).astype(np.float64), synth.bf16_bits_to_f32(exact).astype(np.float64)
+        one_ulp = np.exp2(np.floor(np.log2(np.maximum(np.maximum(np.abs(c64), np.abs(e64)), 2.0 ** -100))) - 7.0)
+        # the accumulated small noise, plus the one bf16 step by which it can move a rounding
+        assert np.all(np.abs(c64 - e64) <= 6 * cfg["sigma_small"] * np.sqrt(step) + one_ulp), "only accumulated small noise"
+    assert 0 < ever_sent.sum() < n

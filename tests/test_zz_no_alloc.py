@@ -15,6 +15,7 @@ import pytest
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
+import oracle
 from paper_2604_14561_b200 import binding, synth
 
 
@@ -64,6 +65,32 @@ def test_static_scratch_matches_workspace_call_twice_in_a_row():
         assert int(want.n_active.item()) == S // T - n_groups * int(np.floor(r * (S // T // n_groups)))
         for name, a, b in zip(("metric", "mask", "idx", "n_active", "v_compact"), want.tensors(), got.tensors()):
             assert torch.equal(a, b), f"{name} differs from the workspace-taking entry point"
+        # and directly against the CPU oracle's rule
+        m_ref = oracle.vmajor_metric(prev.cpu().numpy().view(np.uint16).reshape(S, H, D),
+                                     cur.cpu().numpy().view(np.uint16).reshape(S, H, D), P, T)
+        mask_ref, idx_ref, na_ref = oracle.vmajor_select(m_ref, n_groups, r)
+        assert np.array_equal(got.metric.cpu().numpy().view(np.uint64), m_ref)
+        assert int(got.n_active.item()) == na_ref and np.array_equal(got.mask.cpu().numpy(), mask_ref)
+        assert np.array_equal(got.idx.cpu().numpy()[:na_ref], idx_ref)
+
+
+def test_static_scratch_at_its_unit_limit():
+    """Exactly STATIC_MAX_UNITS per-token units in one group: the largest call the
+    entry point accepts, checked against the oracle."""
+    P, S, H, D, T, r = 2, binding.STATIC_MAX_UNITS, 2, 32, 1, 0.8
+    prev, cur = _inputs(S, H, D, T, 3)
+    got = _Outputs(S, H, D, T)
+    for _ in range(2):
+        binding.vmajor_select_compact_static(prev, cur, P, S, H, D, T, r, 1, *got.tensors())
+    torch.cuda.synchronize()
+    m_ref = oracle.vmajor_metric(prev.cpu().numpy().view(np.uint16).reshape(S, H, D),
+                                 cur.cpu().numpy().view(np.uint16).reshape(S, H, D), P, T)
+    mask_ref, idx_ref, na_ref = oracle.vmajor_select(m_ref, 1, r)
+    assert np.array_equal(got.metric.cpu().numpy().view(np.uint64), m_ref)
+    assert int(got.n_active.item()) == na_ref and np.array_equal(got.mask.cpu().numpy(), mask_ref)
+    assert np.array_equal(got.idx.cpu().numpy()[:na_ref], idx_ref)
+    comp_ref = oracle.pack_active(cur.cpu().numpy().view(np.uint16).reshape(S, H, D), idx_ref, P, T)
+    assert np.array_equal(got.v_compact.cpu().numpy().view(np.uint16)[:comp_ref.size], comp_ref.reshape(-1))
 
 
 def test_static_scratch_refuses_more_units_than_it_holds():
