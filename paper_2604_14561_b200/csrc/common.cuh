@@ -122,7 +122,7 @@ MetricPlan plan_metric(int n_units, long long unit_vecs);
 // Units up to this count are selected by every block of the consuming kernel
 // itself (no selection launch); it is also the largest group the counting
 // selection kernel takes.
-constexpr int kCountMax = 512;
+constexpr int kCountMax = 256;
 
 cudaError_t launch_tapa_phase2(const TapaParams &p, cudaStream_t stream);
 cudaError_t launch_move(const MoveParams &p, cudaStream_t stream);

@@ -16,6 +16,8 @@
 // no one-block stage between the metric pass and the data movement); an active
 // row is then read once and written twice, to the compact send buffer and to its
 // slot of the cached head-parallel tensor.
+#include <mutex>
+
 #include "move_rows.cuh"
 #include "vmajor.cuh"
 
@@ -46,7 +48,8 @@ __global__ void __launch_bounds__(kThreads, kMinBlocks) move_rows_kernel(const _
 
 template <int LPR, bool PAD>
 __global__ void __launch_bounds__(kThreads, kMinBlocks)
-selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constant__ SelectParams sel, const int select_here) {
+selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constant__ SelectParams sel, const int select_here,
+                      const unsigned n_items) {
     __shared__ vmajor::SmallSel sm;
     if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -60,7 +63,10 @@ selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constan
     }
     int n_valid = nv < (long long)p.n_slots ? (int)nv : p.n_slots;
     if (n_valid < 0) n_valid = 0;
-    move_block<LPR, PAD, KIND_MIXED, 4, 4, kThreads, true>(p, blockIdx.x, list, n_valid);
+    // one resident wave of blocks walks the (head range, tensor, token tile) items, so that a
+    // block ranks the units once however many items it moves
+    for (unsigned item = blockIdx.x; item < n_items; item += gridDim.x)
+        move_block<LPR, PAD, KIND_MIXED, 4, 4, kThreads, true>(p, item, list, n_valid);
 }
 
 template <typename K, typename... Args>
@@ -77,6 +83,20 @@ cudaError_t launch_grid(K kernel, long long blocks, cudaStream_t stream, int pdl
     cfg.attrs = attr;
     cfg.numAttrs = (pdl & PDL_LAUNCH_ATTR) ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+// multiprocessors of the current device (looked up once per device)
+int sm_count() {
+    static std::mutex mu;
+    static int count[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    std::lock_guard<std::mutex> lock(mu);
+    if (count[dev] == 0) {
+        int n = 0;
+        count[dev] = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+    }
+    return count[dev];
 }
 
 long long grid_blocks(MoveParams &p, int lpr, int heads_per_block) {
@@ -103,11 +123,22 @@ cudaError_t launch_lpr(MoveParams p, cudaStream_t stream) {
     return launch_grid(move_rows_kernel<LPR, PAD, KIND_MIXED, 4, 4>, grid_blocks(p, LPR, 12), stream, p.pdl, p);
 }
 
+#ifndef COCODIFF_SEL_HEADS
+#define COCODIFF_SEL_HEADS 6
+#endif
 template <int LPR, bool PAD>
 cudaError_t launch_selective_lpr(MoveParams p, const SelectParams *sel, cudaStream_t stream) {
     static const SelectParams none = {};
-    return launch_grid(selective_move_kernel<LPR, PAD>, grid_blocks(p, LPR, 8), stream, p.pdl, p, sel ? *sel : none,
-                       sel ? 1 : 0);
+    // items of 6 heads: fine enough to balance one resident wave (4 blocks on each SM)
+    const long long items = grid_blocks(p, LPR, COCODIFF_SEL_HEADS);
+    if (items > 0xffffffffLL) return cudaErrorInvalidConfiguration;
+#ifdef COCODIFF_SEL_NONPERSISTENT
+    const long long wave = items;
+#else
+    const long long wave = (long long)sm_count() * kMinBlocks;
+#endif
+    return launch_grid(selective_move_kernel<LPR, PAD>, items < wave ? items : wave, stream, p.pdl, p, sel ? *sel : none,
+                       sel ? 1 : 0, (unsigned)items);
 }
 
 // D = 8 * lanes; a lane group is padded to the next power of two.

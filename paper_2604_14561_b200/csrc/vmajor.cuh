@@ -76,12 +76,12 @@ struct SmallSel {
     unsigned long long m[kCountMax];
     int idx[kCountMax];
     unsigned char active[kCountMax];
-    int warp_sums[33];
+    unsigned words[kCountMax / 32];   // the active flags, one bit per unit
 };
 
 template <int BLOCK>
 __device__ int select_small(const SelectParams &p, const int base, const int cnt, SmallSel &sm, const bool publish) {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31;
     for (int e = tid; e < cnt; e += BLOCK) sm.m[e] = unit_metric(p, base + e);
     __syncthreads();
     for (int e = tid; e < cnt; e += BLOCK) {
@@ -95,15 +95,21 @@ __device__ int select_small(const SelectParams &p, const int base, const int cnt
         sm.active[e] = rank >= p.n_cached ? 1 : 0;
     }
     __syncthreads();
-    const int per = (cnt + BLOCK - 1) / BLOCK;
-    const int e_lo = tid * per < cnt ? tid * per : cnt;
-    const int e_hi = e_lo + per < cnt ? e_lo + per : cnt;
-    int c = 0;
-    for (int e = e_lo; e < e_hi; ++e) c += sm.active[e];
-    int total;
-    int pos = block_excl_scan<BLOCK>(c, &total, sm.warp_sums);
-    for (int e = e_lo; e < e_hi; ++e)
-        if (sm.active[e]) sm.idx[pos++] = base + e;
+    const int cnt_pad = (cnt + 31) / 32 * 32;
+    for (int e = tid; e < cnt_pad; e += BLOCK) {
+        const unsigned w = __ballot_sync(0xffffffffu, e < cnt && sm.active[e]);
+        if (lane == 0) sm.words[e >> 5] = w;
+    }
+    __syncthreads();
+    // position of an active unit in the ascending list: the set bits before it
+    int total = 0;
+    for (int w = 0; w < cnt_pad / 32; ++w) total += __popc(sm.words[w]);
+    for (int e = tid; e < cnt; e += BLOCK)
+        if (sm.active[e]) {
+            int pos = __popc(sm.words[e >> 5] & ((1u << (e & 31)) - 1u));
+            for (int w = 0; w < (e >> 5); ++w) pos += __popc(sm.words[w]);
+            sm.idx[pos] = base + e;
+        }
     __syncthreads();
     if (publish) {
         const int out_base = (base / p.g) * (p.g - p.n_cached);
@@ -123,15 +129,17 @@ __device__ int select_small(const SelectParams &p, const int base, const int cnt
 // Large group: one block finds the metric of rank n_cached-1 (mstar) and how
 // many of the units equal to it are cached (t_c), then emits mask and list.
 //
-// Stage 1 (groups of at most 65535 units): a histogram over a 16-bit monotone
-// key of the 64-bit metric - position of the leading one (6 bits) and the ten
-// bits below it - held in shared memory as 65536 16-bit counters.  A scan of the
-// histogram gives the key that contains the wanted rank.  Stage 2 resolves the
-// rank among the units of that key: by counting when they are few, else by
-// 8-bit radix passes over the bits the key does not cover.  Groups beyond 65535
-// units skip stage 1 and run the radix passes over all bits in use.
+// The group's metrics are first copied to shared memory (when they fit), so
+// that every later pass reads them there.  Stage 1 (groups of at most 65535
+// units): a histogram over a monotone key of the 64-bit metric - position of the
+// leading one (6 bits) and the mb bits below it - held in shared memory as
+// 16-bit counters; mb (8..10) is the widest that fits beside the metrics.  A scan
+// of the histogram gives the key that contains the wanted rank.  Stage 2
+// resolves the rank among the units of that key: by counting when they are few,
+// else by 8-bit radix passes over the bits the key does not cover.  Groups
+// beyond 65535 units skip stage 1 and run the radix passes over all bits in use.
 constexpr int kLargeBlock = 1024;
-constexpr int kCandMax = 1024;
+constexpr int kCandMax = 256;
 
 struct LargeSel {
     int warp_sums[33];
@@ -142,35 +150,38 @@ struct LargeSel {
     unsigned long long slots[kLargeBlock / 32];
     unsigned long long cand_val[kCandMax];
     int cand_idx[kCandMax];
+    unsigned less_mask[2048], tie_mask[2048];  // one bit per unit, groups of at most 65536 units
 };
-// dynamic shared memory: 65536 16-bit counters, reused as 32 per-warp 256-bin histograms
-constexpr size_t kLargeDynBytes = 65536 * 2;
+// Dynamic shared memory: [histogram of (64 << mb) 16-bit counters, at least 32 KB - it is
+// reused as 32 per-warp 256-bin histograms by the radix passes][the staged metrics].
+constexpr size_t kLargeDynMax = 200 * 1024;   // beside the static part: inside the 227 KB a block may use
+__host__ __device__ constexpr size_t large_hist_bytes(int mb) { return ((size_t)64 << mb) * 2; }
 
-__device__ __forceinline__ unsigned key16(unsigned long long v) {
+__device__ __forceinline__ unsigned key_of(unsigned long long v, int mb) {
     if (v < 2) return 0;  // 0 and 1 share the first key
     const int e = 63 - __clzll((long long)v);
     const unsigned long long frac = (v << (63 - e)) << 1;  // bits below the leading one, left-aligned
-    return ((unsigned)e << 10) | (unsigned)(frac >> 54);
+    return ((unsigned)e << mb) | (unsigned)(frac >> (64 - mb));
 }
 // smallest metric with that key
-__device__ __forceinline__ unsigned long long key16_base(unsigned key) {
+__device__ __forceinline__ unsigned long long key_base(unsigned key, int mb) {
     if (key == 0) return 0ull;
-    const int e = (int)(key >> 10);
-    const unsigned long long top = 1024ull | (key & 1023u);  // leading one and ten bits
-    return e >= 10 ? top << (e - 10) : top >> (10 - e);
+    const int e = (int)(key >> mb);
+    const unsigned long long top = (1ull << mb) | (key & ((1u << mb) - 1u));  // leading one and mb bits
+    return e >= mb ? top << (e - mb) : top >> (mb - e);
 }
 // number of low bits of the metric that the key leaves open
-__device__ __forceinline__ int key16_low_bits(unsigned key) {
+__device__ __forceinline__ int key_low_bits(unsigned key, int mb) {
     if (key == 0) return 1;
-    const int e = (int)(key >> 10);
-    return e > 10 ? e - 10 : 0;
+    const int e = (int)(key >> mb);
+    return e > mb ? e - mb : 0;
 }
 
 // 8-bit radix passes from `shift_top` down to 0 over the units with
-// key16 == want_key (want_key < 0: all units); k = wanted rank among them.
+// key == want_key (want_key < 0: all units); k = wanted rank among them.
 // Leaves the selected low bits in *prefix_out and the rank among equals in *k_out.
 template <int BLOCK>
-__device__ void radix_passes(const unsigned long long *vals, int g, int want_key, int shift_top, int k,
+__device__ void radix_passes(const unsigned long long *vals, int g, int want_key, int mb, int shift_top, int k,
                              LargeSel &sm, int *warp_hist, unsigned long long *prefix_out, int *k_out) {
     const int tid = threadIdx.x, warp = tid >> 5;
     unsigned long long prefix = 0, pmask = 0;
@@ -180,7 +191,7 @@ __device__ void radix_passes(const unsigned long long *vals, int g, int want_key
         __syncthreads();
         for (int e = tid; e < g; e += BLOCK) {
             const unsigned long long v = vals[e];
-            if ((want_key < 0 || key16(v) == (unsigned)want_key) && (v & pmask) == prefix)
+            if ((want_key < 0 || key_of(v, mb) == (unsigned)want_key) && (v & pmask) == prefix)
                 atomicAdd(&my_hist[(int)((v >> shift) & 255ull)], 1);
         }
         __syncthreads();
@@ -202,9 +213,65 @@ __device__ void radix_passes(const unsigned long long *vals, int g, int want_key
 
 // Threshold form of the rule: unit e is cached iff vals[e] < mstar, or
 // vals[e] == mstar and fewer than t_c units equal to mstar precede it.  Every
-// warp owns a contiguous range of units and walks it 32 at a time (coalesced
-// loads, ballots for the running counts), so two block scans suffice to emit
-// the mask and the ascending list.
+// warp owns a contiguous range of 32-unit chunks.  The metrics are compared once:
+// the "less" and "tie" bits of a chunk are kept as two words in shared memory,
+// and the two counting passes and the writing pass work on those words only
+// (two block scans in all).  For groups of at most 65536 units.
+template <int BLOCK>
+__device__ void emit_selection_masks(const SelectParams &p, int grp, const unsigned long long *vals, bool none,
+                                     unsigned long long mstar, int t_c, LargeSel &sm) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int WARPS = BLOCK / 32;
+    const int g = p.g, base = grp * g, out_base = grp * (g - p.n_cached);
+    const int n_chunks = (g + 31) / 32;
+    const int cpw = (n_chunks + WARPS - 1) / WARPS;
+    const int c_lo = warp * cpw < n_chunks ? warp * cpw : n_chunks;
+    const int c_hi = c_lo + cpw < n_chunks ? c_lo + cpw : n_chunks;
+    const unsigned lt = (1u << lane) - 1u;
+    int ties = 0;
+    for (int c = c_lo; c < c_hi; ++c) {
+        const int e = 32 * c + lane;
+        const unsigned long long v = e < g ? vals[e] : ~0ull;
+        const unsigned lm = __ballot_sync(0xffffffffu, !none && e < g && v < mstar);
+        const unsigned tm = __ballot_sync(0xffffffffu, !none && e < g && v == mstar);
+        if (lane == 0) { sm.less_mask[c] = lm; sm.tie_mask[c] = tm; }
+        ties += __popc(tm);
+    }
+    int scan_total;
+    int tie_rank = block_excl_scan<BLOCK>(lane == 0 ? ties : 0, &scan_total, sm.warp_sums);
+    tie_rank = __shfl_sync(0xffffffffu, tie_rank, 0);
+    // active bits of every chunk (they replace the "less" bits), counted
+    int actives = 0;
+    for (int c = c_lo; c < c_hi; ++c) {
+        const unsigned lm = sm.less_mask[c], tm = sm.tie_mask[c];
+        const unsigned valid = 32 * c + 32 <= g ? 0xffffffffu : ((1u << (g - 32 * c)) - 1u);
+        const bool tie_cached = ((tm >> lane) & 1u) && tie_rank + __popc(tm & lt) < t_c;
+        const unsigned cached = lm | __ballot_sync(0xffffffffu, tie_cached);
+        const unsigned am = ~cached & valid;
+        __syncwarp();
+        if (lane == 0) sm.less_mask[c] = am;
+        actives += __popc(am);
+        tie_rank += __popc(tm);
+    }
+    int pos = block_excl_scan<BLOCK>(lane == 0 ? actives : 0, &scan_total, sm.warp_sums);
+    pos = __shfl_sync(0xffffffffu, pos, 0);
+    for (int c = c_lo; c < c_hi; ++c) {
+        const unsigned am = sm.less_mask[c];
+        const int e = 32 * c + lane;
+        const bool active = (am >> lane) & 1u;
+        if (e < g && COCODIFF_IN_BOUNDS(base + e >= 0 && base + e < p.n, p.debug)) p.mask[base + e] = active ? 1 : 0;
+        if (active) {
+            const int o = out_base + pos + __popc(am & lt);
+            if (COCODIFF_IN_BOUNDS(o >= 0 && o < p.n, p.debug)) p.idx[o] = base + e;
+        }
+        pos += __popc(am);
+    }
+    if (grp == 0 && tid == 0) *p.n_active = p.n_groups * (g - p.n_cached);
+    __syncthreads();
+}
+
+// The same rule for groups of any size: nothing is kept between the passes, the
+// metrics are read and compared in each of them.
 template <int BLOCK>
 __device__ void emit_selection(const SelectParams &p, int grp, const unsigned long long *vals, bool none,
                                unsigned long long mstar, int t_c, int *warp_sums) {
@@ -262,58 +329,79 @@ __device__ void emit_selection(const SelectParams &p, int grp, const unsigned lo
 }
 
 template <int BLOCK>
-__device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm, unsigned *dyn) {
+__device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm, unsigned *dyn, const int mb,
+                                   const int staged) {
     const int tid = threadIdx.x;
     const int g = p.g, n_cached = p.n_cached;
     const bool none = n_cached == 0;
+    const int hist_words = (int)(large_hist_bytes(mb) / 4);
     // the group's metrics; pieces are summed once and kept in metric_out
-    const unsigned long long *vals;
-    if (p.parts == 0) vals = p.metric + (long long)grp * g;
+    const unsigned long long *gvals;
+    if (p.parts == 0) gvals = p.metric + (long long)grp * g;
     else {
         for (int e = tid; e < g; e += BLOCK) p.metric_out[(long long)grp * g + e] = unit_metric(p, grp * g + e);
         __syncthreads();  // this block reads back only what it wrote itself
-        vals = p.metric_out + (long long)grp * g;
+        gvals = p.metric_out + (long long)grp * g;
+    }
+    const unsigned long long *vals = gvals;
+    if (staged) {
+        // copy to shared memory, four independent loads in flight per thread
+        unsigned long long *sv = reinterpret_cast<unsigned long long *>(dyn + hist_words);
+        for (int e = tid; e < g; e += 4 * BLOCK) {
+            unsigned long long v[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) v[i] = e + i * BLOCK < g ? __ldcg(gvals + e + i * BLOCK) : 0ull;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (e + i * BLOCK < g) sv[e + i * BLOCK] = v[i];
+        }
+        vals = sv;
     }
     if (!none) {
         int *warp_hist = reinterpret_cast<int *>(dyn);
         const int k = n_cached - 1;
         if (g <= 65535) {
-            // stage 1: 16-bit key histogram, two counters per 32-bit word
-            for (int i = tid; i < 32768; i += BLOCK) dyn[i] = 0;
-            __syncthreads();
+            // stage 1: key histogram, two 16-bit counters per 32-bit word
+            for (int i = tid; i < hist_words; i += BLOCK) dyn[i] = 0;
+            __syncthreads();  // also publishes the staged metrics
             for (int e = tid; e < g; e += BLOCK) {
-                const unsigned key = key16(vals[e]);
+                const unsigned key = key_of(vals[e], mb);
                 atomicAdd(&dyn[key >> 1], (key & 1u) ? 0x10000u : 1u);
             }
             __syncthreads();
-            // every thread owns 64 consecutive keys (32 words)
+            // every thread owns a run of consecutive keys
+            // (read in a rotated order: consecutive lanes then touch different banks)
+            const int wpt = hist_words / BLOCK;  // words per thread: 8, 16 or 32
             unsigned cnt = 0;
-            for (int i = 0; i < 32; ++i) { const unsigned w = dyn[tid * 32 + i]; cnt += (w & 0xffffu) + (w >> 16); }
+            for (int i = 0; i < wpt; ++i) {
+                const unsigned w = dyn[tid * wpt + ((i + tid) & (wpt - 1))];
+                cnt += (w & 0xffffu) + (w >> 16);
+            }
             int total;
             const int excl = block_excl_scan<BLOCK>((int)cnt, &total, sm.warp_sums);
             if (cnt > 0 && excl <= k && k < excl + (int)cnt) {
                 int run = excl;
-                for (int i = 0; i < 64; ++i) {
-                    const unsigned w = dyn[tid * 32 + (i >> 1)];
+                for (int i = 0; i < 2 * wpt; ++i) {
+                    const unsigned w = dyn[tid * wpt + (i >> 1)];
                     const int c = (int)((i & 1) ? (w >> 16) : (w & 0xffffu));
-                    if (k < run + c) { sm.sel_bin = tid * 64 + i; sm.sel_k = k - run; sm.n_cand = c; break; }
+                    if (k < run + c) { sm.sel_bin = tid * 2 * wpt + i; sm.sel_k = k - run; sm.n_cand = c; break; }
                     run += c;
                 }
             }
             __syncthreads();
             const unsigned bin = (unsigned)sm.sel_bin;
             const int kk = sm.sel_k, n_cand = sm.n_cand;
-            const int low_bits = key16_low_bits(bin);
+            const int low_bits = key_low_bits(bin, mb);
             __syncthreads();
             if (low_bits == 0) {
-                if (tid == 0) { sm.mstar = key16_base(bin); sm.t_c = kk + 1; }
+                if (tid == 0) { sm.mstar = key_base(bin, mb); sm.t_c = kk + 1; }
             } else if (n_cand <= kCandMax) {
                 // stage 2a: rank the few units of that key by counting
                 if (tid == 0) sm.n_cand = 0;
                 __syncthreads();
                 for (int e = tid; e < g; e += BLOCK) {
                     const unsigned long long v = vals[e];
-                    if (key16(v) == bin) {
+                    if (key_of(v, mb) == bin) {
                         const int slot = atomicAdd(&sm.n_cand, 1);
                         if (slot < kCandMax) { sm.cand_val[slot] = v; sm.cand_idx[slot] = e; }
                     }
@@ -335,11 +423,11 @@ __device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm,
                 // stage 2b: radix passes over the bits below the key
                 unsigned long long prefix;
                 int k_eq;
-                radix_passes<BLOCK>(vals, g, (int)bin, 8 * ((low_bits - 1) / 8), kk, sm, warp_hist, &prefix, &k_eq);
+                radix_passes<BLOCK>(vals, g, (int)bin, mb, 8 * ((low_bits - 1) / 8), kk, sm, warp_hist, &prefix, &k_eq);
                 if (tid == 0) {
                     const int covered = 8 * ((low_bits - 1) / 8) + 8;
                     const unsigned long long lowmask = covered >= 64 ? ~0ull : ((1ull << covered) - 1ull);
-                    sm.mstar = (key16_base(bin) & ~lowmask) | prefix;
+                    sm.mstar = (key_base(bin, mb) & ~lowmask) | prefix;
                     sm.t_c = k_eq + 1;
                 }
             }
@@ -351,12 +439,13 @@ __device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm,
             while (top > 0 && (mx >> top) == 0ull) top -= 8;
             unsigned long long prefix;
             int k_eq;
-            radix_passes<BLOCK>(vals, g, -1, top, k, sm, warp_hist, &prefix, &k_eq);
+            radix_passes<BLOCK>(vals, g, -1, mb, top, k, sm, warp_hist, &prefix, &k_eq);
             if (tid == 0) { sm.mstar = prefix; sm.t_c = k_eq + 1; }
         }
-        __syncthreads();
     }
-    emit_selection<BLOCK>(p, grp, vals, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm.warp_sums);
+    __syncthreads();
+    if (g <= 65536) emit_selection_masks<BLOCK>(p, grp, vals, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm);
+    else emit_selection<BLOCK>(p, grp, vals, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm.warp_sums);
 }
 
 // ---------------------------------------------------------------------------

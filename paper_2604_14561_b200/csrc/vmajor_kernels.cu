@@ -31,12 +31,12 @@ __global__ void __launch_bounds__(256) vmajor_select_small_kernel(const __grid_c
 }
 
 __global__ void __launch_bounds__(kLargeBlock)
-vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int pdl) {
+vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int mb, const int staged, const int pdl) {
     __shared__ LargeSel sm;
-    extern __shared__ unsigned dyn_words[];
+    extern __shared__ __align__(16) unsigned dyn_words[];
     if (pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
-    select_group_large<kLargeBlock>(p, blockIdx.x, sm, dyn_words);
+    select_group_large<kLargeBlock>(p, blockIdx.x, sm, dyn_words, mb, staged);
 }
 
 __global__ void __launch_bounds__(kMetricThreads, kMetricBlocksPerSm)
@@ -123,7 +123,7 @@ cudaError_t launch_select(const SelectParams &p, cudaStream_t stream, int pdl) {
     if (p.n == 0) return cudaMemsetAsync(p.n_active, 0, sizeof(int32_t), stream);
     if (p.g <= kCountMax)
         return launch_maybe_programmatic(vmajor_select_small_kernel, dim3(p.n_groups), dim3(256), 0, stream, pdl, p, pdl);
-    // the 128 KB of dynamic shared memory need the opt-in, once per device
+    // the dynamic shared memory needs the opt-in, once per device
     static std::mutex mu;
     static bool attr_set[64] = {};
     int dev = 0;
@@ -134,13 +134,20 @@ cudaError_t launch_select(const SelectParams &p, cudaStream_t stream, int pdl) {
         std::lock_guard<std::mutex> lock(mu);
         if (!attr_set[dev]) {
             e = cudaFuncSetAttribute(vmajor_select_large_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)kLargeDynBytes);
+                                     (int)kLargeDynMax);
             if (e != cudaSuccess) return e;
             attr_set[dev] = true;
         }
     }
-    return launch_maybe_programmatic(vmajor_select_large_kernel, dim3(p.n_groups), dim3(kLargeBlock), kLargeDynBytes,
-                                     stream, pdl, p, pdl);
+    // the widest key histogram that leaves room for the group's metrics; without room
+    // for both the metrics stay in global memory and the histogram takes its full width
+    const size_t vals_bytes = (size_t)p.g * sizeof(unsigned long long);
+    int mb = p.g <= 4096 ? 8 : 10, staged = 1;  // few units: a narrow histogram is cleared and scanned faster
+    while (mb > 8 && large_hist_bytes(mb) + vals_bytes > kLargeDynMax) --mb;
+    if (large_hist_bytes(mb) + vals_bytes > kLargeDynMax) { mb = 10; staged = 0; }
+    const size_t dyn = large_hist_bytes(mb) + (staged ? vals_bytes : 0);
+    return launch_maybe_programmatic(vmajor_select_large_kernel, dim3(p.n_groups), dim3(kLargeBlock), dyn, stream, pdl,
+                                     p, mb, staged, pdl);
 }
 
 cudaError_t launch_metric(const MetricParams &p, cudaStream_t stream) {
