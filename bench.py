@@ -683,6 +683,15 @@ def next_rows(torch, binding, args):
         torch.cuda.synchronize()
     per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(total)]
     full = [binding.cache_schedule(i, total, warmup, interval)[0] for i in range(total)]
+    # the stand-alone compaction and the receiver-only scatter of 29 of 144 units (the selective step
+    # itself moves its rows in one fused pass; these calls launch a worst-case grid because the host
+    # does not know n_active, and the blocks beyond the active units return at once)
+    binding.vmajor_select_compact(v, v, P, S, H, D, T, 0.8, 1, metric, mask, idx, na, None, ws, ws_bytes, stream=sq)
+    torch.cuda.synchronize()
+    moved = 6 * int(na.item()) * T * H * D * 2
+    timed("pack_active_qkv_standalone", lambda: binding.pack_active_qkv(q, k, v, wq, wk, cfg["eps"], cs, idx, na, *comp,
+                                                                         P, S, H, D, T, stream=sq), moved)
+    timed("unpack_qkv_receiver_only", lambda: binding.unpack_qkv(*comp, idx, na, qh, kh, vh, P, S, H, D, T, stream=sq), moved)
     out["schedule_50_steps"] = {
         "total_us": 1e3 * sum(per_step), "always_full_us_estimate": 1e3 * total * statistics.mean(t for t, f in zip(per_step, full) if f),
         "full_steps": sum(full), "us_full_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if f),

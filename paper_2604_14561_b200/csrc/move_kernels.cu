@@ -123,20 +123,13 @@ cudaError_t launch_lpr(MoveParams p, cudaStream_t stream) {
     return launch_grid(move_rows_kernel<LPR, PAD, KIND_MIXED, 4, 4>, grid_blocks(p, LPR, 12), stream, p.pdl, p);
 }
 
-#ifndef COCODIFF_SEL_HEADS
-#define COCODIFF_SEL_HEADS 6
-#endif
 template <int LPR, bool PAD>
 cudaError_t launch_selective_lpr(MoveParams p, const SelectParams *sel, cudaStream_t stream) {
     static const SelectParams none = {};
     // items of 6 heads: fine enough to balance one resident wave (4 blocks on each SM)
-    const long long items = grid_blocks(p, LPR, COCODIFF_SEL_HEADS);
+    const long long items = grid_blocks(p, LPR, 6);
     if (items > 0xffffffffLL) return cudaErrorInvalidConfiguration;
-#ifdef COCODIFF_SEL_NONPERSISTENT
-    const long long wave = items;
-#else
     const long long wave = (long long)sm_count() * kMinBlocks;
-#endif
     return launch_grid(selective_move_kernel<LPR, PAD>, items < wave ? items : wave, stream, p.pdl, p, sel ? *sel : none,
                        sel ? 1 : 0, (unsigned)items);
 }

@@ -129,21 +129,22 @@ __device__ int select_small(const SelectParams &p, const int base, const int cnt
 // Large group: one block finds the metric of rank n_cached-1 (mstar) and how
 // many of the units equal to it are cached (t_c), then emits mask and list.
 //
-// The group's metrics are first copied to shared memory (when they fit), so
-// that every later pass reads them there.  Stage 1 (groups of at most 65535
-// units): a histogram over a monotone key of the 64-bit metric - position of the
-// leading one (6 bits) and the mb bits below it - held in shared memory as
-// 16-bit counters; mb (8..10) is the widest that fits beside the metrics.  A scan
-// of the histogram gives the key that contains the wanted rank.  Stage 2
-// resolves the rank among the units of that key: by counting when they are few,
-// else by 8-bit radix passes over the bits the key does not cover.  Groups
-// beyond 65535 units skip stage 1 and run the radix passes over all bits in use.
+// Groups of at most 65535 units: one pass over the metrics computes a monotone
+// key of each 64-bit metric - position of its leading one (6 bits) and the mb
+// bits below it (mb = 10, or 9 when that does not fit) -, keeps the keys in
+// shared memory as 16-bit values and counts them in a histogram of 16-bit
+// counters.  A scan of the histogram gives the key that contains the wanted
+// rank; every later pass reads the 2-byte keys and fetches the 8-byte metric
+// again only for the few units of that key.  The rank among those units is
+// resolved by counting when they are few, else by 8-bit radix passes over the
+// bits the key does not cover.  Larger groups skip the keys and run the radix
+// passes over all bits in use, reading the metrics from global memory.
 constexpr int kLargeBlock = 1024;
 constexpr int kCandMax = 256;
 
 struct LargeSel {
     int warp_sums[33];
-    int sel_bin, sel_k;
+    int sel_bin, sel_k, sel_owner;
     unsigned long long mstar;
     int t_c;
     int n_cand;
@@ -151,10 +152,11 @@ struct LargeSel {
     unsigned long long cand_val[kCandMax];
     int cand_idx[kCandMax];
     unsigned less_mask[2048], tie_mask[2048];  // one bit per unit, groups of at most 65536 units
+    int chunk_pos[2048];                       // active units before each 32-unit chunk
 };
 // Dynamic shared memory: [histogram of (64 << mb) 16-bit counters, at least 32 KB - it is
-// reused as 32 per-warp 256-bin histograms by the radix passes][the staged metrics].
-constexpr size_t kLargeDynMax = 200 * 1024;   // beside the static part: inside the 227 KB a block may use
+// reused as 32 per-warp 256-bin histograms by the radix passes][one 16-bit key per unit].
+constexpr size_t kLargeDynMax = 196 * 1024;   // beside the static part: inside the 227 KB a block may use
 __host__ __device__ constexpr size_t large_hist_bytes(int mb) { return ((size_t)64 << mb) * 2; }
 
 __device__ __forceinline__ unsigned key_of(unsigned long long v, int mb) {
@@ -177,12 +179,13 @@ __device__ __forceinline__ int key_low_bits(unsigned key, int mb) {
     return e > mb ? e - mb : 0;
 }
 
-// 8-bit radix passes from `shift_top` down to 0 over the units with
-// key == want_key (want_key < 0: all units); k = wanted rank among them.
-// Leaves the selected low bits in *prefix_out and the rank among equals in *k_out.
+// 8-bit radix passes from `shift_top` down to 0 over the units whose key is
+// want_key (keys == nullptr: all units); k = wanted rank among them.  Leaves the
+// selected low bits in *prefix_out and the rank among equals in *k_out.
 template <int BLOCK>
-__device__ void radix_passes(const unsigned long long *vals, int g, int want_key, int mb, int shift_top, int k,
-                             LargeSel &sm, int *warp_hist, unsigned long long *prefix_out, int *k_out) {
+__device__ void radix_passes(const unsigned long long *vals, const unsigned short *keys, int g, unsigned want_key,
+                             int shift_top, int k, LargeSel &sm, int *warp_hist, unsigned long long *prefix_out,
+                             int *k_out) {
     const int tid = threadIdx.x, warp = tid >> 5;
     unsigned long long prefix = 0, pmask = 0;
     int *my_hist = warp_hist + warp * 256;
@@ -190,9 +193,9 @@ __device__ void radix_passes(const unsigned long long *vals, int g, int want_key
         for (int i = tid; i < (BLOCK / 32) * 256; i += BLOCK) warp_hist[i] = 0;
         __syncthreads();
         for (int e = tid; e < g; e += BLOCK) {
-            const unsigned long long v = vals[e];
-            if ((want_key < 0 || key_of(v, mb) == (unsigned)want_key) && (v & pmask) == prefix)
-                atomicAdd(&my_hist[(int)((v >> shift) & 255ull)], 1);
+            if (keys != nullptr && keys[e] != want_key) continue;
+            const unsigned long long v = __ldcg(vals + e);
+            if ((v & pmask) == prefix) atomicAdd(&my_hist[(int)((v >> shift) & 255ull)], 1);
         }
         __syncthreads();
         int c = 0;
@@ -212,59 +215,73 @@ __device__ void radix_passes(const unsigned long long *vals, int g, int want_key
 }
 
 // Threshold form of the rule: unit e is cached iff vals[e] < mstar, or
-// vals[e] == mstar and fewer than t_c units equal to mstar precede it.  Every
-// warp owns a contiguous range of 32-unit chunks.  The metrics are compared once:
-// the "less" and "tie" bits of a chunk are kept as two words in shared memory,
-// and the two counting passes and the writing pass work on those words only
-// (two block scans in all).  For groups of at most 65536 units.
+// vals[e] == mstar and fewer than t_c units equal to mstar precede it.  The
+// metrics are compared once: the "less" and "tie" bits of every 32-unit chunk
+// are kept as two words in shared memory.  Then one thread per chunk turns them
+// into the chunk's active bits (two block scans over the chunks give the number
+// of ties and of active units before each chunk), and a last pass over the units
+// writes mask and list.  No pass carries a running count from one iteration to
+// the next.  For groups of at most 65536 units.
 template <int BLOCK>
-__device__ void emit_selection_masks(const SelectParams &p, int grp, const unsigned long long *vals, bool none,
-                                     unsigned long long mstar, int t_c, LargeSel &sm) {
+__device__ void emit_selection_masks(const SelectParams &p, int grp, const unsigned long long *vals,
+                                     const unsigned short *keys, unsigned bin, bool none, unsigned long long mstar,
+                                     int t_c, LargeSel &sm) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int WARPS = BLOCK / 32;
     const int g = p.g, base = grp * g, out_base = grp * (g - p.n_cached);
     const int n_chunks = (g + 31) / 32;
-    const int cpw = (n_chunks + WARPS - 1) / WARPS;
-    const int c_lo = warp * cpw < n_chunks ? warp * cpw : n_chunks;
-    const int c_hi = c_lo + cpw < n_chunks ? c_lo + cpw : n_chunks;
-    const unsigned lt = (1u << lane) - 1u;
-    int ties = 0;
-    for (int c = c_lo; c < c_hi; ++c) {
+    for (int c = warp; c < n_chunks; c += WARPS) {
         const int e = 32 * c + lane;
-        const unsigned long long v = e < g ? vals[e] : ~0ull;
-        const unsigned lm = __ballot_sync(0xffffffffu, !none && e < g && v < mstar);
-        const unsigned tm = __ballot_sync(0xffffffffu, !none && e < g && v == mstar);
+        bool less = false, tie = false;
+        if (!none && e < g) {
+            const unsigned key = keys[e];  // a key below / above the selected one decides without the metric
+            less = key < bin;
+            if (key == bin) {
+                const unsigned long long v = __ldcg(vals + e);
+                less = v < mstar;
+                tie = v == mstar;
+            }
+        }
+        const unsigned lm = __ballot_sync(0xffffffffu, less);
+        const unsigned tm = __ballot_sync(0xffffffffu, tie);
         if (lane == 0) { sm.less_mask[c] = lm; sm.tie_mask[c] = tm; }
-        ties += __popc(tm);
     }
+    __syncthreads();
+    // thread t owns chunks 2t and 2t+1 (n_chunks <= 2 * BLOCK)
+    unsigned lm[2] = {0, 0}, tm[2] = {0, 0}, am[2] = {0, 0};
+    for (int i = 0; i < 2; ++i)
+        if (2 * tid + i < n_chunks) { lm[i] = sm.less_mask[2 * tid + i]; tm[i] = sm.tie_mask[2 * tid + i]; }
     int scan_total;
-    int tie_rank = block_excl_scan<BLOCK>(lane == 0 ? ties : 0, &scan_total, sm.warp_sums);
-    tie_rank = __shfl_sync(0xffffffffu, tie_rank, 0);
-    // active bits of every chunk (they replace the "less" bits), counted
-    int actives = 0;
-    for (int c = c_lo; c < c_hi; ++c) {
-        const unsigned lm = sm.less_mask[c], tm = sm.tie_mask[c];
-        const unsigned valid = 32 * c + 32 <= g ? 0xffffffffu : ((1u << (g - 32 * c)) - 1u);
-        const bool tie_cached = ((tm >> lane) & 1u) && tie_rank + __popc(tm & lt) < t_c;
-        const unsigned cached = lm | __ballot_sync(0xffffffffu, tie_cached);
-        const unsigned am = ~cached & valid;
-        __syncwarp();
-        if (lane == 0) sm.less_mask[c] = am;
-        actives += __popc(am);
-        tie_rank += __popc(tm);
+    int tie_rank = block_excl_scan<BLOCK>(__popc(tm[0]) + __popc(tm[1]), &scan_total, sm.warp_sums);
+    for (int i = 0; i < 2; ++i) {
+        const int c = 2 * tid + i;
+        if (c < n_chunks) {
+            // the first (t_c - tie_rank) ties of the chunk are cached
+            unsigned tie_cached = 0, rest = tm[i];
+            for (int left = t_c - tie_rank; left > 0 && rest != 0; --left) { tie_cached |= rest & (0u - rest); rest &= rest - 1u; }
+            const unsigned valid = 32 * c + 32 <= g ? 0xffffffffu : ((1u << (g - 32 * c)) - 1u);
+            am[i] = ~(lm[i] | tie_cached) & valid;
+            tie_rank += __popc(tm[i]);
+        }
     }
-    int pos = block_excl_scan<BLOCK>(lane == 0 ? actives : 0, &scan_total, sm.warp_sums);
-    pos = __shfl_sync(0xffffffffu, pos, 0);
-    for (int c = c_lo; c < c_hi; ++c) {
-        const unsigned am = sm.less_mask[c];
+    int pos = block_excl_scan<BLOCK>(__popc(am[0]) + __popc(am[1]), &scan_total, sm.warp_sums);
+    for (int i = 0; i < 2; ++i)
+        if (2 * tid + i < n_chunks) {
+            sm.less_mask[2 * tid + i] = am[i];
+            sm.chunk_pos[2 * tid + i] = pos;
+            pos += __popc(am[i]);
+        }
+    __syncthreads();
+    const unsigned lt = (1u << lane) - 1u;
+    for (int c = warp; c < n_chunks; c += WARPS) {
+        const unsigned a = sm.less_mask[c];
         const int e = 32 * c + lane;
-        const bool active = (am >> lane) & 1u;
+        const bool active = (a >> lane) & 1u;
         if (e < g && COCODIFF_IN_BOUNDS(base + e >= 0 && base + e < p.n, p.debug)) p.mask[base + e] = active ? 1 : 0;
         if (active) {
-            const int o = out_base + pos + __popc(am & lt);
+            const int o = out_base + sm.chunk_pos[c] + __popc(a & lt);
             if (COCODIFF_IN_BOUNDS(o >= 0 && o < p.n, p.debug)) p.idx[o] = base + e;
         }
-        pos += __popc(am);
     }
     if (grp == 0 && tid == 0) *p.n_active = p.n_groups * (g - p.n_cached);
     __syncthreads();
@@ -329,48 +346,51 @@ __device__ void emit_selection(const SelectParams &p, int grp, const unsigned lo
 }
 
 template <int BLOCK>
-__device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm, unsigned *dyn, const int mb,
-                                   const int staged) {
-    const int tid = threadIdx.x;
+__device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm, unsigned *dyn, const int mb) {
+    const int tid = threadIdx.x, lane = tid & 31;
     const int g = p.g, n_cached = p.n_cached;
     const bool none = n_cached == 0;
-    const int hist_words = (int)(large_hist_bytes(mb) / 4);
     // the group's metrics; pieces are summed once and kept in metric_out
-    const unsigned long long *gvals;
-    if (p.parts == 0) gvals = p.metric + (long long)grp * g;
+    const unsigned long long *vals;
+    if (p.parts == 0) vals = p.metric + (long long)grp * g;
     else {
         for (int e = tid; e < g; e += BLOCK) p.metric_out[(long long)grp * g + e] = unit_metric(p, grp * g + e);
-        __syncthreads();  // this block reads back only what it wrote itself
-        gvals = p.metric_out + (long long)grp * g;
+        __threadfence();
+        __syncthreads();  // this block reads back (from the L2) only what it wrote itself
+        vals = p.metric_out + (long long)grp * g;
     }
-    const unsigned long long *vals = gvals;
-    if (staged) {
-        // copy to shared memory, four independent loads in flight per thread
-        unsigned long long *sv = reinterpret_cast<unsigned long long *>(dyn + hist_words);
-        for (int e = tid; e < g; e += 4 * BLOCK) {
-            unsigned long long v[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) v[i] = e + i * BLOCK < g ? __ldcg(gvals + e + i * BLOCK) : 0ull;
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (e + i * BLOCK < g) sv[e + i * BLOCK] = v[i];
-        }
-        vals = sv;
-    }
+    const bool keyed = g <= 65535;
+    const int hist_words = (int)(large_hist_bytes(mb) / 4);
+    unsigned short *keys = reinterpret_cast<unsigned short *>(dyn + hist_words);
+    unsigned bin = 0;
     if (!none) {
         int *warp_hist = reinterpret_cast<int *>(dyn);
         const int k = n_cached - 1;
-        if (g <= 65535) {
-            // stage 1: key histogram, two 16-bit counters per 32-bit word
+        if (keyed) {
+            // one pass over the metrics (sixteen loads in flight per thread, the first batch
+            // issued before the histogram is cleared): keys and their histogram
+            constexpr int UL = 16;
+            unsigned long long v[UL];
+#pragma unroll
+            for (int u = 0; u < UL; ++u) v[u] = tid + u * BLOCK < g ? __ldcg(vals + tid + u * BLOCK) : 0ull;
             for (int i = tid; i < hist_words; i += BLOCK) dyn[i] = 0;
-            __syncthreads();  // also publishes the staged metrics
-            for (int e = tid; e < g; e += BLOCK) {
-                const unsigned key = key_of(vals[e], mb);
-                atomicAdd(&dyn[key >> 1], (key & 1u) ? 0x10000u : 1u);
+            __syncthreads();
+            for (int e0 = tid; e0 < g; e0 += UL * BLOCK) {
+                if (e0 != tid) {
+#pragma unroll
+                    for (int u = 0; u < UL; ++u) v[u] = e0 + u * BLOCK < g ? __ldcg(vals + e0 + u * BLOCK) : 0ull;
+                }
+#pragma unroll
+                for (int u = 0; u < UL; ++u)
+                    if (e0 + u * BLOCK < g) {
+                        const unsigned key = key_of(v[u], mb);
+                        keys[e0 + u * BLOCK] = (unsigned short)key;
+                        atomicAdd(&dyn[key >> 1], (key & 1u) ? 0x10000u : 1u);
+                    }
             }
             __syncthreads();
-            // every thread owns a run of consecutive keys
-            // (read in a rotated order: consecutive lanes then touch different banks)
+            // every thread owns a run of consecutive keys (read in a rotated order: consecutive
+            // lanes then touch different banks)
             const int wpt = hist_words / BLOCK;  // words per thread: 8, 16 or 32
             unsigned cnt = 0;
             for (int i = 0; i < wpt; ++i) {
@@ -379,33 +399,44 @@ __device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm,
             }
             int total;
             const int excl = block_excl_scan<BLOCK>((int)cnt, &total, sm.warp_sums);
-            if (cnt > 0 && excl <= k && k < excl + (int)cnt) {
-                int run = excl;
-                for (int i = 0; i < 2 * wpt; ++i) {
-                    const unsigned w = dyn[tid * wpt + (i >> 1)];
-                    const int c = (int)((i & 1) ? (w >> 16) : (w & 0xffffu));
-                    if (k < run + c) { sm.sel_bin = tid * 2 * wpt + i; sm.sel_k = k - run; sm.n_cand = c; break; }
-                    run += c;
+            if (cnt > 0 && excl <= k && k < excl + (int)cnt) { sm.sel_owner = tid; sm.sel_k = k - excl; }
+            __syncthreads();
+            // the first warp walks the winning thread's run: lane l takes word l
+            if (tid < 32) {
+                const int owner = sm.sel_owner, kk0 = sm.sel_k;
+                __syncwarp();
+                const unsigned w = lane < wpt ? dyn[owner * wpt + lane] : 0u;
+                const int lo = (int)(w & 0xffffu), hi = (int)(w >> 16);
+                int incl = lo + hi;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const int t = __shfl_up_sync(0xffffffffu, incl, off);
+                    if (lane >= off) incl += t;
+                }
+                const int before = incl - lo - hi;
+                if (before <= kk0 && kk0 < incl) {
+                    const bool in_hi = kk0 >= before + lo;
+                    sm.sel_bin = (owner * wpt + lane) * 2 + (in_hi ? 1 : 0);
+                    sm.sel_k = kk0 - before - (in_hi ? lo : 0);
+                    sm.n_cand = in_hi ? hi : lo;
                 }
             }
             __syncthreads();
-            const unsigned bin = (unsigned)sm.sel_bin;
+            bin = (unsigned)sm.sel_bin;
             const int kk = sm.sel_k, n_cand = sm.n_cand;
             const int low_bits = key_low_bits(bin, mb);
             __syncthreads();
             if (low_bits == 0) {
                 if (tid == 0) { sm.mstar = key_base(bin, mb); sm.t_c = kk + 1; }
             } else if (n_cand <= kCandMax) {
-                // stage 2a: rank the few units of that key by counting
+                // the few units of that key: fetched again and ranked by counting
                 if (tid == 0) sm.n_cand = 0;
                 __syncthreads();
-                for (int e = tid; e < g; e += BLOCK) {
-                    const unsigned long long v = vals[e];
-                    if (key_of(v, mb) == bin) {
+                for (int e = tid; e < g; e += BLOCK)
+                    if (keys[e] == bin) {
                         const int slot = atomicAdd(&sm.n_cand, 1);
-                        if (slot < kCandMax) { sm.cand_val[slot] = v; sm.cand_idx[slot] = e; }
+                        if (slot < kCandMax) { sm.cand_val[slot] = __ldcg(vals + e); sm.cand_idx[slot] = e; }
                     }
-                }
                 __syncthreads();
                 for (int i = tid; i < n_cand; i += BLOCK) {
                     const unsigned long long my = sm.cand_val[i];
@@ -420,10 +451,10 @@ __device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm,
                     if (rank == kk) { sm.mstar = my; sm.t_c = ties_before + 1; }
                 }
             } else {
-                // stage 2b: radix passes over the bits below the key
+                // many units of that key: radix passes over the bits below the key
                 unsigned long long prefix;
                 int k_eq;
-                radix_passes<BLOCK>(vals, g, (int)bin, mb, 8 * ((low_bits - 1) / 8), kk, sm, warp_hist, &prefix, &k_eq);
+                radix_passes<BLOCK>(vals, keys, g, bin, 8 * ((low_bits - 1) / 8), kk, sm, warp_hist, &prefix, &k_eq);
                 if (tid == 0) {
                     const int covered = 8 * ((low_bits - 1) / 8) + 8;
                     const unsigned long long lowmask = covered >= 64 ? ~0ull : ((1ull << covered) - 1ull);
@@ -433,18 +464,18 @@ __device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm,
             }
         } else {
             unsigned long long mx = 0;
-            for (int e = tid; e < g; e += BLOCK) { const unsigned long long v = vals[e]; mx = v > mx ? v : mx; }
+            for (int e = tid; e < g; e += BLOCK) { const unsigned long long v = __ldcg(vals + e); mx = v > mx ? v : mx; }
             mx = block_max_u64<BLOCK>(mx, sm.slots);
             int top = 56;
             while (top > 0 && (mx >> top) == 0ull) top -= 8;
             unsigned long long prefix;
             int k_eq;
-            radix_passes<BLOCK>(vals, g, -1, mb, top, k, sm, warp_hist, &prefix, &k_eq);
+            radix_passes<BLOCK>(vals, nullptr, g, 0u, top, k, sm, warp_hist, &prefix, &k_eq);
             if (tid == 0) { sm.mstar = prefix; sm.t_c = k_eq + 1; }
         }
     }
     __syncthreads();
-    if (g <= 65536) emit_selection_masks<BLOCK>(p, grp, vals, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm);
+    if (keyed) emit_selection_masks<BLOCK>(p, grp, vals, keys, bin, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm);
     else emit_selection<BLOCK>(p, grp, vals, none, none ? 0ull : sm.mstar, none ? 0 : sm.t_c, sm.warp_sums);
 }
 

@@ -31,12 +31,12 @@ __global__ void __launch_bounds__(256) vmajor_select_small_kernel(const __grid_c
 }
 
 __global__ void __launch_bounds__(kLargeBlock)
-vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int mb, const int staged, const int pdl) {
+vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int mb, const int pdl) {
     __shared__ LargeSel sm;
     extern __shared__ __align__(16) unsigned dyn_words[];
     if (pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
-    select_group_large<kLargeBlock>(p, blockIdx.x, sm, dyn_words, mb, staged);
+    select_group_large<kLargeBlock>(p, blockIdx.x, sm, dyn_words, mb);
 }
 
 __global__ void __launch_bounds__(kMetricThreads, kMetricBlocksPerSm)
@@ -139,15 +139,14 @@ cudaError_t launch_select(const SelectParams &p, cudaStream_t stream, int pdl) {
             attr_set[dev] = true;
         }
     }
-    // the widest key histogram that leaves room for the group's metrics; without room
-    // for both the metrics stay in global memory and the histogram takes its full width
-    const size_t vals_bytes = (size_t)p.g * sizeof(unsigned long long);
-    int mb = p.g <= 4096 ? 8 : 10, staged = 1;  // few units: a narrow histogram is cleared and scanned faster
-    while (mb > 8 && large_hist_bytes(mb) + vals_bytes > kLargeDynMax) --mb;
-    if (large_hist_bytes(mb) + vals_bytes > kLargeDynMax) { mb = 10; staged = 0; }
-    const size_t dyn = large_hist_bytes(mb) + (staged ? vals_bytes : 0);
-    return launch_maybe_programmatic(vmajor_select_large_kernel, dim3(p.n_groups), dim3(kLargeBlock), dyn, stream, pdl,
-                                     p, mb, staged, pdl);
+    // groups of up to 65535 units keep one 16-bit key per unit behind the histogram; the
+    // histogram has 256, 512 or 1024 keys per leading-one position: a narrow one is cleared
+    // and scanned faster, a wide one leaves fewer units to tell apart afterwards
+    const size_t keys_bytes = p.g <= 65535 ? ((size_t)p.g * 2 + 15) / 16 * 16 : 0;
+    int mb = p.g <= 4096 ? 8 : (p.g <= 16384 ? 9 : 10);
+    if (large_hist_bytes(mb) + keys_bytes > kLargeDynMax) mb = 9;
+    return launch_maybe_programmatic(vmajor_select_large_kernel, dim3(p.n_groups), dim3(kLargeBlock),
+                                     large_hist_bytes(mb) + keys_bytes, stream, pdl, p, mb, pdl);
 }
 
 cudaError_t launch_metric(const MetricParams &p, cudaStream_t stream) {
