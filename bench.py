@@ -247,6 +247,38 @@ def time_graph(torch, fn, stream, steps, flush=None):
         return None
 
 
+def time_graph_loop(torch, fn, stream, calls, replays):
+    """`calls` consecutive calls of `fn` captured into one CUDA graph (no host work between the
+    launches), replayed `replays` times between two events; ms per call, median of 5; None if
+    capture is refused."""
+    try:
+        for _ in range(calls):
+            fn()
+        stream.synchronize()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(calls):
+                fn()
+        torch.cuda.synchronize()
+        out = []
+        with torch.cuda.stream(stream):
+            g.replay()
+            for _ in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                for _ in range(replays):
+                    g.replay()
+                b.record(stream)
+                stream.synchronize()
+                out.append(a.elapsed_time(b) / (replays * calls))
+        torch.cuda.synchronize()
+        return statistics.median(out)
+    except Exception as exc:
+        sys.stderr.write(f"graph capture skipped: {exc}\n")
+        return None
+
+
 def max_over_ranks(ms, world, device):
     """The slowest rank's time: every multi-GPU number is the max over ranks."""
     if world <= 1:
@@ -531,11 +563,32 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
             cold = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 3, flush=flush))
             warm = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 3))
             out[name][oname] = {"us_cold_l2": 1e3 * cold, "gbs_effective_cold_l2": b / (cold * 1e-3) / 1e9,
-                                "gbs_effective_above_launch_floor": b / max(1e3 * cold - floor, 1e-3) / 1e3,
                                 "us_warm_l2": 1e3 * warm}
             gr = time_graph(torch, lambda: full(order), sq, iters, flush=flush)
             if gr is not None:
                 out[name][oname]["us_cold_l2_cuda_graph"] = 1e3 * statistics.median(gr)
+        if name != "temporal":
+            # Layers back to back on rotating buffer sets: no event or flush between the calls, and
+            # the sets together exceed four times the L2 (when memory allows), so that every call
+            # reads from HBM and the write-back of its output falls inside the timed region.
+            n_sets = max(2, min(64, int(np.ceil(4 * 126e6 / b)) + 1))
+            sets = [([t.clone() for t in (q, k, v)], [torch.empty_like(qh) for _ in range(3)]) for _ in range(n_sets)]
+            for oname, order in (("v_first", binding.V_FIRST), ("lump", binding.LUMP)):
+                calls = [0]
+
+                def rotating():
+                    (a, c, d), (x, y, z) = sets[calls[0] % n_sets]
+                    calls[0] += 1
+                    binding.prologue(a, c, d, x, y, z, wq, wk, cfg["eps"], cs, P, S, H, D, order=order,
+                                     stream_qk=sq, stream_v=sv)
+                ms = time_graph_loop(torch, rotating, sq, n_sets, replays=10)
+                if ms is None:
+                    continue
+                out[name][oname]["back_to_back_rotating_buffers"] = {
+                    "us_per_layer": 1e3 * ms, "gbs": b / (ms * 1e-3) / 1e9, "buffer_sets": n_sets,
+                    "how": "one CUDA graph of buffer_sets consecutive calls, replayed 10 times between two events (median of 5)",
+                    "working_set_bytes": n_sets * b, "exceeds_4x_l2": bool(n_sets * b >= 4 * 126e6)}
+            del sets
         del q, k, v, qh, kh, vh
     return out
 
@@ -624,7 +677,7 @@ def temporal_rows(torch, binding, args):
     return out
 
 
-def next_rows(torch, binding, args):
+def next_rows(torch, binding, args, rows=("inverse", "tapa", "schedule", "moves")):
     """Rows beyond the headline path, on the temporal workload (P=24, S=9216, H=24, D=128):
     inverse exchange, the two TAPA phases, and the paper's 50-step cache schedule (5 warm-up
     steps, refresh every 10 steps, linear cache ratio)."""
@@ -649,14 +702,16 @@ def next_rows(torch, binding, args):
         out[name] = {"us_cold_l2": 1e3 * t, "bytes": nbytes, "gbs": nbytes / (t * 1e-3) / 1e9}
 
     binding.prologue(q, k, v, qh, kh, vh, wq, wk, cfg["eps"], cs, P, S, H, D, order=binding.LUMP, stream_qk=sq, stream_v=sq)
-    back = [new() for _ in range(3)]
-    timed("inverse_a2a", lambda: binding.ulysses_a2a_inverse(qh, kh, vh, *back, P, S, H, D, stream=sq), 6 * E * 2)
-    del back
-    p1 = [new(2) for _ in range(3)]
-    th = [new() for _ in range(3)]
-    timed("tapa_phase1", lambda: binding.tapa_phase1(q, k, v, *p1, P, S, H, D, stream=sq), 12 * E * 2)
-    timed("tapa_phase2", lambda: binding.tapa_phase2(*p1, *th, P, S, H, D, stream=sq), 6 * E * 2)
-    del p1, th
+    if "inverse" in rows:
+        back = [new() for _ in range(3)]
+        timed("inverse_a2a", lambda: binding.ulysses_a2a_inverse(qh, kh, vh, *back, P, S, H, D, stream=sq), 6 * E * 2)
+        del back
+    if "tapa" in rows:
+        p1 = [new(2) for _ in range(3)]
+        th = [new() for _ in range(3)]
+        timed("tapa_phase1", lambda: binding.tapa_phase1(q, k, v, *p1, P, S, H, D, stream=sq), 12 * E * 2)
+        timed("tapa_phase2", lambda: binding.tapa_phase2(*p1, *th, P, S, H, D, stream=sq), 6 * E * 2)
+        del p1, th
 
     comp = [new() for _ in range(3)]
 
@@ -669,20 +724,28 @@ def next_rows(torch, binding, args):
     mask = torch.zeros(n, dtype=torch.uint8, device="cuda")
     idx = torch.zeros(n, dtype=torch.int32, device="cuda")
     na = torch.zeros(1, dtype=torch.int32, device="cuda")
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(total + 1)]
-    for rep in range(2):                 # first pass warms up
-        sent = []
-        torch.cuda.synchronize()
-        ev[0].record(sq)
-        for step_i in range(total):
-            _, s_el = binding.layer_step(step_i, total, warmup, interval, v, q, k, v, wq, wk,
-                                         cfg["eps"], cs, P, S, H, D, T, 1, metric, mask, idx, na, comp[0], comp[1],
-                                         comp[2], qh, kh, vh, ws, ws_bytes, order=binding.LUMP, stream_qk=sq, stream_v=sq)
-            sent.append(s_el)
-            ev[step_i + 1].record(sq)
-        torch.cuda.synchronize()
-    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(total)]
-    full = [binding.cache_schedule(i, total, warmup, interval)[0] for i in range(total)]
+    if "schedule" in rows:
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(total + 1)]
+        for rep in range(2):                 # first pass warms up
+            sent = []
+            torch.cuda.synchronize()
+            ev[0].record(sq)
+            for step_i in range(total):
+                _, s_el = binding.layer_step(step_i, total, warmup, interval, v, q, k, v, wq, wk,
+                                             cfg["eps"], cs, P, S, H, D, T, 1, metric, mask, idx, na, comp[0], comp[1],
+                                             comp[2], qh, kh, vh, ws, ws_bytes, order=binding.LUMP, stream_qk=sq, stream_v=sq)
+                sent.append(s_el)
+                ev[step_i + 1].record(sq)
+            torch.cuda.synchronize()
+        per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(total)]
+        full = [binding.cache_schedule(i, total, warmup, interval)[0] for i in range(total)]
+        out["schedule_50_steps"] = {
+            "total_us": 1e3 * sum(per_step), "always_full_us_estimate": 1e3 * total * statistics.mean(t for t, f in zip(per_step, full) if f),
+            "full_steps": sum(full), "us_full_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if f),
+            "us_selective_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if not f),
+            "exchanged_fraction_of_always_full": sum(sent) / (total * 3 * E), "l2": "warm (steps back to back)"}
+    if "moves" not in rows:
+        return out
     # the stand-alone compaction and the receiver-only scatter of 29 of 144 units (the selective step
     # itself moves its rows in one fused pass; these calls launch a worst-case grid because the host
     # does not know n_active, and the blocks beyond the active units return at once)
@@ -692,11 +755,6 @@ def next_rows(torch, binding, args):
     timed("pack_active_qkv_standalone", lambda: binding.pack_active_qkv(q, k, v, wq, wk, cfg["eps"], cs, idx, na, *comp,
                                                                          P, S, H, D, T, stream=sq), moved)
     timed("unpack_qkv_receiver_only", lambda: binding.unpack_qkv(*comp, idx, na, qh, kh, vh, P, S, H, D, T, stream=sq), moved)
-    out["schedule_50_steps"] = {
-        "total_us": 1e3 * sum(per_step), "always_full_us_estimate": 1e3 * total * statistics.mean(t for t, f in zip(per_step, full) if f),
-        "full_steps": sum(full), "us_full_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if f),
-        "us_selective_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if not f),
-        "exchanged_fraction_of_always_full": sum(sent) / (total * 3 * E), "l2": "warm (steps back to back)"}
     return out
 
 
@@ -711,6 +769,8 @@ def main():
     ap.add_argument("--only-temporal", action="store_true",
                     help="run only the temporal workload (its eight steps, then the rows beyond the headline path), for profiling")
     ap.add_argument("--no-next-rows", action="store_true", help="with --only-temporal: the eight steps only")
+    ap.add_argument("--rows", nargs="+", default=None, choices=["steps", "inverse", "tapa", "schedule", "moves"],
+                    help="with --only-temporal: only these parts (short launch lists for profiling)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -718,9 +778,11 @@ def main():
         import torch
         from paper_2604_14561_b200 import binding
         torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-        pc = {"temporal_steps": temporal_rows(torch, binding, args)}
+        pc = {}
+        if args.rows is None or "steps" in args.rows:
+            pc["temporal_steps"] = temporal_rows(torch, binding, args)
         if not args.no_next_rows:
-            pc["next_rows_temporal"] = next_rows(torch, binding, args)
+            pc["next_rows_temporal"] = next_rows(torch, binding, args, *([tuple(args.rows)] if args.rows else []))
         print(json.dumps({"per_config": pc}, ensure_ascii=False))
     else:
         run_ours(args)

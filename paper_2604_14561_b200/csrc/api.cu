@@ -302,7 +302,7 @@ int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint
                  int H, int D, int T, cudaStream_t st) {
     MoveParams p = make_pack_params(in, out, nullptr, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T);
     if (p.njobs == 0) return COCODIFF_OK;
-    CK(launch_move(p, st));
+    CK(launch_selective_move(p, nullptr, st));  // a resident wave that walks the active tiles only
     return COCODIFF_OK;
 }
 
@@ -351,7 +351,7 @@ int enqueue_unpack(const uint16_t *const in[3], uint16_t *const out[3], const in
                    const int32_t *n_active, int slots, int S, int H, int D, int T, cudaStream_t st) {
     MoveParams p = make_unpack_params(in, out, idx, n_active, slots, S, H, D, T);
     if (p.njobs == 0) return COCODIFF_OK;
-    CK(launch_move(p, st));
+    CK(launch_selective_move(p, nullptr, st));  // a resident wave that walks the active tiles only
     return COCODIFF_OK;
 }
 

@@ -48,8 +48,7 @@ __global__ void __launch_bounds__(kThreads, kMinBlocks) move_rows_kernel(const _
 
 template <int LPR, bool PAD>
 __global__ void __launch_bounds__(kThreads, kMinBlocks)
-selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constant__ SelectParams sel, const int select_here,
-                      const unsigned n_items) {
+selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constant__ SelectParams sel, const int select_here) {
     __shared__ vmajor::SmallSel sm;
     if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -63,10 +62,17 @@ selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constan
     }
     int n_valid = nv < (long long)p.n_slots ? (int)nv : p.n_slots;
     if (n_valid < 0) n_valid = 0;
-    // one resident wave of blocks walks the (head range, tensor, token tile) items, so that a
-    // block ranks the units once however many items it moves
-    for (unsigned item = blockIdx.x; item < n_items; item += gridDim.x)
-        move_block<LPR, PAD, KIND_MIXED, 4, 4, kThreads, true>(p, item, list, n_valid);
+    // One resident wave of blocks walks the (head range, tensor, token tile) items, so that a
+    // block ranks the units once however many items it moves.  Only the tiles that hold active
+    // slots are walked (the grid's capacity may be larger: the host need not know n_active).
+    constexpr unsigned TOK = kThreads / LPR;
+    const unsigned tiles_cap = ((unsigned)p.n_slots + TOK - 1) / TOK;
+    const unsigned tiles = ((unsigned)n_valid + TOK - 1) / TOK;
+    const unsigned groups = (unsigned)p.head_split * (unsigned)p.njobs;   // (head range, tensor) pairs
+    for (unsigned item = blockIdx.x; item < tiles * groups; item += gridDim.x) {
+        const unsigned grp = item / tiles, tile = item - grp * tiles;
+        move_block<LPR, PAD, KIND_MIXED, 4, 4, kThreads, true>(p, grp * tiles_cap + tile, list, n_valid);
+    }
 }
 
 template <typename K, typename... Args>
@@ -131,7 +137,7 @@ cudaError_t launch_selective_lpr(MoveParams p, const SelectParams *sel, cudaStre
     if (items > 0xffffffffLL) return cudaErrorInvalidConfiguration;
     const long long wave = (long long)sm_count() * kMinBlocks;
     return launch_grid(selective_move_kernel<LPR, PAD>, items < wave ? items : wave, stream, p.pdl, p, sel ? *sel : none,
-                       sel ? 1 : 0, (unsigned)items);
+                       sel ? 1 : 0);
 }
 
 // D = 8 * lanes; a lane group is padded to the next power of two.
