@@ -51,6 +51,8 @@ int check_unit(int P, int S, int T) {
 }
 
 // Two timing-less events per (thread, device) for the fork / join of the V stream.
+// (They live as long as the thread's use of the device: destroying them from a thread-exit
+// hook could run after the runtime has shut down.)
 struct ForkJoin {
     cudaEvent_t fork = nullptr, join = nullptr;
 };

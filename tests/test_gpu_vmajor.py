@@ -124,6 +124,39 @@ def test_selection_alone_with_ties_and_wide_keys(n, n_groups):
         assert np.all(idx.cpu().numpy()[na_ref:] == -1)
 
 
+def test_selection_alone_random_shapes():
+    """Seeded random draws of the group structure, the ratio and the shape of the metric
+    distribution: every selection kernel and every branch inside them against the oracle."""
+    rng = np.random.default_rng(2024)
+    for case in range(60):
+        g = int(rng.choice([1, 2, 31, 32, 33, 100, 255, 256, 257, 300, 512, 1000, 2047, 2048, 2049, 4097, 9000, 16385, 40000]))
+        n_groups = int(rng.choice([1, 1, 2, 3, 7])) if g < 20000 else 1
+        n = g * n_groups
+        r = float(rng.choice([0.0, 1.0, rng.random(), rng.random(), 1.0 / g, 1.0 - 1.0 / g]))
+        kind = rng.integers(0, 5)
+        if kind == 0:
+            m = rng.integers(0, 3, n).astype(np.uint64)                                   # almost all ties
+        elif kind == 1:
+            m = rng.integers(0, 2 ** 63, n).astype(np.uint64) * np.uint64(2)              # all 64 bits in use
+        elif kind == 2:
+            m = np.maximum(rng.normal(3.0e5, 4.0e3, n), 0).astype(np.uint64)               # one tight cluster
+        elif kind == 3:
+            m = (np.uint64(1) << rng.integers(0, 60, n).astype(np.uint64)) + rng.integers(0, 2, n).astype(np.uint64)
+        else:
+            m = np.full(n, int(rng.integers(0, 2 ** 40)), np.uint64)                      # all equal
+            m[rng.integers(0, n, max(1, n // 10))] += np.uint64(1)
+        mask = torch.full((n,), 9, dtype=torch.uint8, device="cuda")
+        idx = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+        na = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+        binding.vmajor_select(dev(m), n, r, n_groups, mask, idx, na)
+        torch.cuda.synchronize()
+        mask_ref, idx_ref, na_ref = oracle.vmajor_select(m, n_groups, r)
+        what = (case, g, n_groups, r, int(kind))
+        assert int(na.item()) == na_ref, what
+        assert np.array_equal(mask.cpu().numpy(), mask_ref), what
+        assert np.array_equal(idx.cpu().numpy()[:na_ref], idx_ref), what
+
+
 @pytest.mark.parametrize("P,S,H,D,T", [(2, 256, 4, 64, 16), (4, 512, 4, 128, 1), (3, 99, 3, 32, 11), (2, 384, 2, 256, 64)])
 def test_pack_active_qk_and_unpack(P, S, H, D, T):
     rng = np.random.default_rng(S)
