@@ -118,7 +118,8 @@ def test_empty_sequence_is_a_no_op():
     assert np.all(out.host() == 0x5A5A)
 
 
-@pytest.mark.parametrize("P,S,H,D", [(2, 256, 4, 64), (4, 1000, 8, 128), (1, 77, 5, 32)])
+@pytest.mark.parametrize("P,S,H,D", [(2, 256, 4, 64), (4, 1000, 8, 128), (1, 77, 5, 32),
+                                      (24, 9216, 24, 128)])      # the size the benchmark times the inverse at
 def test_exchange_bit_exact_bijection_and_skips(P, S, H, D):
     L, cfg = _layer(P, S, H, D, seed=7)
     E = S * H * D

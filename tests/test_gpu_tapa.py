@@ -15,7 +15,8 @@ from gpu_util import Guarded, dev, u16
 
 
 @pytest.mark.parametrize("P,S,H,D", [(2, 256, 4, 64), (4, 1000, 8, 128), (12, 1752, 24, 128), (6, 66, 6, 32), (8, 320, 16, 256),
-                                      (2, 130, 4, 96), (4, 36, 4, 8), (2, 50, 2, 200)])
+                                      (2, 130, 4, 96), (4, 36, 4, 8), (2, 50, 2, 200),
+                                      (24, 9216, 24, 128)])      # the size the benchmark times
 def test_two_phases_match_oracle_and_flat_exchange(P, S, H, D):
     E = S * H * D
     x = {t: synth.normal_bf16(3, t, E).reshape(S, H, D) for t in "qkv"}

@@ -248,10 +248,16 @@ def test_temporal_steps_select_compact_unpack(small):
         assert np.array_equal(metric, m_ref) and np.array_equal(mask, mask_ref)
         assert na == na_ref and np.array_equal(idx, idx_ref)
         assert np.array_equal(idx, hot), "active set = the strongly perturbed tiles"
-        for x, w, w_np in (("k", wk, seq.wk), ("q", wq, seq.wq)):
-            binding.pack_active(d[x], w, cfg["eps"], cs, sel.idx, sel.n_active, comp[x].t, P, S, H, D, T)
-        for x, src in (("v", sel.v_compact), ("k", comp["k"]), ("q", comp["q"])):
-            binding.unpack(src.t, sel.idx, sel.n_active, cache[x].t, P, S, H, D, T)
+        if step % 2:      # one tensor per call
+            for x, w, w_np in (("k", wk, seq.wk), ("q", wq, seq.wq)):
+                binding.pack_active(d[x], w, cfg["eps"], cs, sel.idx, sel.n_active, comp[x].t, P, S, H, D, T)
+            for x, src in (("v", sel.v_compact), ("k", comp["k"]), ("q", comp["q"])):
+                binding.unpack(src.t, sel.idx, sel.n_active, cache[x].t, P, S, H, D, T)
+        else:             # the batched calls
+            binding.pack_active_qkv(d["q"], d["k"], None, wq, wk, cfg["eps"], cs, sel.idx, sel.n_active,
+                                    comp["q"].t, comp["k"].t, None, P, S, H, D, T)
+            binding.unpack_qkv(comp["q"].t, comp["k"].t, sel.v_compact.t, sel.idx, sel.n_active,
+                               cache["q"].t, cache["k"].t, cache["v"].t, P, S, H, D, T)
         torch.cuda.synchronize()
         # oracle: norm + RoPE on all rows, extract the active ones, scatter
         oracle.unpack(oracle.pack_active(cur["v"], idx_ref, P, T), idx_ref, cache_ref["v"], P, T)
