@@ -72,27 +72,69 @@ __device__ __forceinline__ unsigned long long unit_metric(const SelectParams &p,
 // counting (metric, index) pairs in shared memory; the units of rank >= n_cached
 // are active.  Leaves the ascending active list in sm.idx and returns its
 // length; with publish the block also writes metric_out, mask, idx and n_active.
+constexpr int kStageMax = 768;   // piece sums staged at once (units * pieces of the selections that run in a consumer)
 struct SmallSel {
     unsigned long long m[kCountMax];
+    unsigned long long stage[kStageMax];
     int idx[kCountMax];
     unsigned char active[kCountMax];
     unsigned words[kCountMax / 32];   // the active flags, one bit per unit
+    int wide;                         // some metric does not leave room for the index beside it
 };
 
 template <int BLOCK>
 __device__ int select_small(const SelectParams &p, const int base, const int cnt, SmallSel &sm, const bool publish) {
     const int tid = threadIdx.x, lane = tid & 31;
-    for (int e = tid; e < cnt; e += BLOCK) sm.m[e] = unit_metric(p, base + e);
-    __syncthreads();
-    for (int e = tid; e < cnt; e += BLOCK) {
-        const int g0 = (e / p.g) * p.g;  // base is a multiple of g
-        const unsigned long long my = sm.m[e];
-        int rank = 0;
-        for (int j = g0; j < g0 + p.g; ++j) {
-            const unsigned long long o = sm.m[j];
-            rank += (o < my) | ((o == my) & (j < e));
+    if (tid == 0) sm.wide = 0;
+    const int n_pieces = cnt * p.parts;
+    if (p.parts >= 2 && n_pieces <= kStageMax) {
+        // the piece sums: coalesced, and all loads of a thread in flight together
+        const unsigned long long *src = p.partial + (long long)base * p.parts;
+        unsigned long long v[(kStageMax + BLOCK - 1) / BLOCK];
+#pragma unroll
+        for (int u = 0; u < (kStageMax + BLOCK - 1) / BLOCK; ++u)
+            v[u] = (tid + u * BLOCK < n_pieces && COCODIFF_IN_BOUNDS((long long)base * p.parts + tid + u * BLOCK < (long long)p.n * p.parts, p.debug))
+                       ? __ldcg(src + tid + u * BLOCK) : 0ull;
+#pragma unroll
+        for (int u = 0; u < (kStageMax + BLOCK - 1) / BLOCK; ++u)
+            if (tid + u * BLOCK < n_pieces) sm.stage[tid + u * BLOCK] = v[u];
+        __syncthreads();
+        for (int e = tid; e < cnt; e += BLOCK) {
+            unsigned long long sum = 0;
+            for (int k = 0; k < p.parts; ++k) sum += sm.stage[e * p.parts + k];
+            sm.m[e] = sum;
         }
-        sm.active[e] = rank >= p.n_cached ? 1 : 0;
+    } else {
+        for (int e = tid; e < cnt; e += BLOCK) sm.m[e] = unit_metric(p, base + e);
+    }
+    __syncthreads();
+    // Rank by counting.  While every metric is below 2^55 the pair (metric, unit) is one 64-bit
+    // key and a rank costs one comparison per other unit; else the two fields are compared.
+    for (int e = tid; e < cnt; e += BLOCK)
+        if (sm.m[e] >> 55) sm.wide = 1;
+    __syncthreads();
+    if (!sm.wide) {
+        for (int e = tid; e < cnt; e += BLOCK) sm.stage[e] = (sm.m[e] << 9) | (unsigned long long)e;  // cnt <= 256 < 2^9
+        __syncthreads();
+        for (int e = tid; e < cnt; e += BLOCK) {
+            const int g0 = (e / p.g) * p.g;  // base is a multiple of g
+            const unsigned long long my = sm.stage[e];
+            int rank = 0;
+#pragma unroll 4
+            for (int j = g0; j < g0 + p.g; ++j) rank += sm.stage[j] < my;
+            sm.active[e] = rank >= p.n_cached ? 1 : 0;
+        }
+    } else {
+        for (int e = tid; e < cnt; e += BLOCK) {
+            const int g0 = (e / p.g) * p.g;
+            const unsigned long long my = sm.m[e];
+            int rank = 0;
+            for (int j = g0; j < g0 + p.g; ++j) {
+                const unsigned long long o = sm.m[j];
+                rank += (o < my) | ((o == my) & (j < e));
+            }
+            sm.active[e] = rank >= p.n_cached ? 1 : 0;
+        }
     }
     __syncthreads();
     const int cnt_pad = (cnt + 31) / 32 * 32;
