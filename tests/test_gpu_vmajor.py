@@ -343,3 +343,69 @@ def test_selective_prologue_one_call(order, two_streams, P, S, H, D, T, r, n_gro
     for t in "qkv":
         assert np.array_equal(comp2[t].host(), comp[t].host())
         assert np.array_equal(cache2[t].host(), cache[t].host())
+
+
+def test_selective_prologue_random_small_shapes():
+    """Seeded random draws of (P, S, H, D, T, r, groups, order): the fused selective step
+    against the oracle on shapes nobody picked by hand."""
+    rng = np.random.default_rng(77)
+    for case in range(36):
+        P = int(rng.choice([1, 2, 3, 4, 6]))
+        H = P * int(rng.integers(1, 4))
+        D = int(rng.choice([8, 16, 24, 32, 48, 64, 96, 128, 160, 256]))
+        T = int(rng.choice([1, 2, 3, 5, 8, 16, 64]))
+        S = P * T * int(rng.integers(1, 40 if T < 16 else 6))
+        n = S // T
+        divisors = [g for g in (1, 2, 3, P, n) if g >= 1 and n % g == 0]
+        n_groups = int(rng.choice(divisors))
+        r = float(rng.choice([0.0, 1.0, 0.5, 0.8, rng.random()]))
+        order, two = [(binding.LUMP, False), (binding.V_FIRST, True), (binding.V_FIRST, False)][case % 3]
+        what = dict(case=case, P=P, S=S, H=H, D=D, T=T, r=r, n_groups=n_groups, order=order, two_streams=two)
+        E = S * H * D
+        prev, cur_v, _ = _pair(S, H, D, T, seed=1000 + case)
+        x = {"q": synth.normal_bf16(20 + case, "q", E).reshape(S, H, D), "k": synth.normal_bf16(20 + case, "k", E).reshape(S, H, D),
+             "v": cur_v}
+        w = {"q": synth.normal_bf16(20 + case, "wq", D, 1.0, 0.1), "k": synth.normal_bf16(20 + case, "wk", D, 1.0, 0.1)}
+        pos = rng.integers(0, 150, (S, 2)).astype(np.int32)
+        cs_ref, cs = oracle.rope_table_2d(pos, D, 10000.0), rope_table(pos, D, 10000.0)
+        old = {t: synth.normal_bf16(9, "old" + t, E).reshape(H, S, D) for t in "qkv"}
+        comp = {t: Guarded(E) for t in "qkv"}
+        cache = {t: Guarded(E, fill=old[t]) for t in "qkv"}
+        sel = Selector(P, S, H, D, T)
+        d = {t: dev(x[t]) for t in "qkv"}
+        sq = torch.cuda.Stream()
+        sv = torch.cuda.Stream() if two else sq
+        torch.cuda.synchronize()
+        binding.selective_prologue(dev(prev), d["q"], d["k"], d["v"], dev(w["q"]), dev(w["k"]), 1e-6, cs, P, S, H, D, T,
+                                   r, n_groups, sel.metric, sel.mask, sel.idx, sel.n_active,
+                                   comp["q"].t, comp["k"].t, comp["v"].t, cache["q"].t, cache["k"].t, cache["v"].t,
+                                   sel.ws, sel.ws_bytes, order=order, stream_qk=sq, stream_v=sv)
+        sq.synchronize()
+        m_ref = oracle.vmajor_metric(prev, cur_v, P, T)
+        mask_ref, idx_ref, na_ref = oracle.vmajor_select(m_ref, n_groups, r)
+        assert np.array_equal(sel.metric.cpu().numpy().view(np.uint64)[:n], m_ref), what
+        assert int(sel.n_active.item()) == na_ref, what
+        assert np.array_equal(sel.mask.cpu().numpy()[:n], mask_ref), what
+        assert np.array_equal(sel.idx.cpu().numpy()[:na_ref], idx_ref), what
+        tok = (idx_ref[:, None] * T + np.arange(T)[None, :]).reshape(-1).astype(np.int64)
+        for t in "qkv":
+            if t == "v":
+                ref, ref_f = x["v"], None
+            else:
+                ref, ref_f = oracle.norm_rope(x[t], w[t], 1e-6, cs_ref, want_f32=True)
+            comp_ref = oracle.pack_active(ref, idx_ref, P, T)
+            got_c = comp[t].host()[:comp_ref.size].reshape(comp_ref.shape)
+            want_cache = oracle.unpack(comp_ref, idx_ref, old[t].copy(), P, T)
+            got_cache = cache[t].host((H, S, D))
+            if t == "v":
+                assert np.array_equal(got_c, comp_ref) and np.array_equal(got_cache, want_cache), what
+            else:
+                if na_ref:
+                    assert_norm_rope_close(got_c, comp_ref, np.ascontiguousarray(ref_f[tok].transpose(1, 0, 2)), f"{t} {what}")
+                    assert np.array_equal(got_cache[:, tok], got_c), what
+                untouched = np.ones(S, bool)
+                untouched[tok] = False
+                assert np.array_equal(got_cache[:, untouched], want_cache[:, untouched]), what
+            assert np.all(comp[t].host()[comp_ref.size:] == 0x5A5A), what
+            comp[t].assert_guards()
+            cache[t].assert_guards()
