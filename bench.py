@@ -667,6 +667,22 @@ def temporal_rows(torch, binding, args):
         "launches_per_step": {"lump": 2, "v_first": 3},
         "kernel_break_out": "per-kernel durations of these same launches: profiles/vmajor_selective_step_temporal.md (ncu)",
         "api": "cocodiff_selective_prologue"}
+    # the metric pass and its selection alone (no compaction follows, so the selection is a launch of
+    # its own), and - for context - a library read-only reduction over the same two tensors
+    def metric_alone():
+        binding.vmajor_select_compact(steps[0]["v"], steps[1]["v"], P, S, H, D, T, r, n_groups, metric, mask, idx, na, None,
+                                      ws, binding.vmajor_workspace_bytes(P, S, H, D, T), stream=sq)
+    sink = torch.zeros(2, dtype=torch.int64, device="cuda")
+
+    def torch_read_only():
+        with torch.cuda.stream(sq):
+            torch.sum(steps[0]["v"].reshape(-1).view(torch.int64), dim=0, keepdim=True, out=sink[0:1])
+            torch.sum(steps[1]["v"].reshape(-1).view(torch.int64), dim=0, keepdim=True, out=sink[1:2])
+    out["metric_pass_context"] = {
+        "bytes": 2 * E * 2,
+        "us_metric_and_selection_alone": 1e3 * statistics.mean(time_steps(torch, metric_alone, sq, iters, 3, flush=flush)),
+        "us_torch_sum_of_the_same_two_tensors": 1e3 * statistics.mean(time_steps(torch, torch_read_only, sq, iters, 3, flush=flush)),
+        "note": "both between two events after an L2 flush; the library reduction (two launches) reads the same 113 MB"}
     gr = time_graph(torch, lambda: selective(1, binding.LUMP), sq, iters, flush=flush)
     if gr is not None:
         out["steps_1_to_7_selective"]["us_step_1_lump_cuda_graph"] = 1e3 * statistics.median(gr)
