@@ -7,6 +7,18 @@ A step is one pass of the prologue over one layer of the 21k-token workload
 (P=12 virtual ranks, S=21024, H=24, D=128, bf16), through the C ABI.  N > 1
 (torchrun) runs N independent replicas, one per GPU: the path has no exchange
 between devices in this build.  Rank 0 prints one JSON line.
+
+Beside the contract's keys the line carries: `repeats` (the headline loop five more
+times, >= 20 ms each), `roofline` (the dominant launch timed back to back),
+`e2e` (host tensors in and out through cocodiff_prologue_host), `cpu_baseline`
+(the oracle on one core, on all cores, and the distance statistics between the
+kernels' and the oracle's results on the sample it ran on) and `per_config`:
+the other workloads (per call after an L2 flush, and back to back on rotating
+buffers), the temporal workload as its eight steps (full step, selective steps,
+per-token units), and the rows beyond the headline path (inverse exchange, the
+two TAPA phases, the 50-step schedule, stand-alone compaction and scatter).
+`--only-main`, `--only-temporal`, `--rows`, `--no-next-rows` cut the run down for
+profiling.
 """
 from __future__ import annotations
 
