@@ -136,6 +136,24 @@ def oracle_all_cores(sub, L, tokens, budget_s=5.0):
             "build": "the same oracle source compiled with -fopenmp", "passes": reps}
 
 
+def oracle_per_config(names=("tiny", "sd3", "qwen768", "temporal")):
+    """ms per layer of the oracle's full prologue on the other workloads: one core, and the
+    OpenMP build on all cores (best of three)."""
+    import oracle
+    out = {}
+    for name in names:
+        cfg = synth.config(name)
+        L = synth.make_layer(cfg)
+        one = min(oracle_sample(cfg, L, cfg["S"]) for _ in range(2))
+        try:
+            oracle.use_all_cores(True)
+            many = min(oracle_sample(cfg, L, cfg["S"]) for _ in range(3))
+        finally:
+            oracle.use_all_cores(False)
+        out[name] = {"ms_one_core": 1e3 * one, "ms_all_cores": 1e3 * many}
+    return out
+
+
 def parity_of_sample(cfg, L, tokens, got_heads, oracle_heads):
     """Distance statistics between the kernels' Q and K and the oracle's on the sample the
     CPU baseline ran on (computed outside every timed region, with the tests' own rule)."""
@@ -478,6 +496,7 @@ def run_ours(args):
                "ms_per_layer_extrapolated": 1e3 * spent / reps * S / tokens,
                "sample": f"{reps} passes over the first {tokens} of {S} tokens (one rank's shard) of the same layer",
                "all_cores": oracle_all_cores(sub, L, tokens),
+               "other_workloads_ms_per_layer": oracle_per_config(),
                "parity_on_sample": parity_of_sample(cfg, L, tokens, got_heads, oracle_heads)}
 
         line = {
@@ -572,10 +591,11 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
         b = algorithmic_bytes(cfg)
         out[name] = {"bytes": b, "fits_in_l2": b < 126e6 * 2}
         for oname, order in (("v_first", binding.V_FIRST), ("lump", binding.LUMP)):
-            cold = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 3, flush=flush))
-            warm = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 3))
-            out[name][oname] = {"us_cold_l2": 1e3 * cold, "gbs_effective_cold_l2": b / (cold * 1e-3) / 1e9,
-                                "us_warm_l2": 1e3 * warm}
+            cold_all = time_steps(torch, lambda: full(order), sq, iters, 10, flush=flush)
+            cold = statistics.median(cold_all)
+            warm = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 10))
+            out[name][oname] = {"us_cold_l2": 1e3 * cold, "us_cold_l2_min": 1e3 * min(cold_all), "iterations": iters,
+                                "gbs_effective_cold_l2": b / (cold * 1e-3) / 1e9, "us_warm_l2": 1e3 * warm}
             gr = time_graph(torch, lambda: full(order), sq, iters, flush=flush)
             if gr is not None:
                 out[name][oname]["us_cold_l2_cuda_graph"] = 1e3 * statistics.median(gr)
