@@ -780,7 +780,8 @@ def next_rows(torch, binding, args, rows=("inverse", "tapa", "schedule", "moves"
     if "tapa" in rows:
         p1 = [new(2) for _ in range(3)]
         th = [new() for _ in range(3)]
-        timed("tapa_phase1", lambda: binding.tapa_phase1(q, k, v, *p1, P, S, H, D, stream=sq), 12 * E * 2)
+        timed("tapa_phase1", lambda: binding.tapa_phase1(q, k, v, *p1, P, S, H, D, stream=sq), 9 * E * 2)
+        out["tapa_phase1"]["note"] = "every shard is read once and written to both rings' holdings: 3 tensors x (1 read + 2 writes)"
         timed("tapa_phase2", lambda: binding.tapa_phase2(*p1, *th, P, S, H, D, stream=sq), 6 * E * 2)
         del p1, th
 

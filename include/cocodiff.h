@@ -244,7 +244,8 @@ int cocodiff_layer_step(int step, int total_steps, int warmup, int sync_interval
  * tile holds all tokens of its GPU.  x_p1 = [2][P/2][2*S/P][H][D], x_p1[t][g] =
  * holdings of tile t of GPU g (2*S*H*D elements per tensor); x_p1[t] as a whole
  * is a [S][H][D] tensor, so V's x_p1[0] can be given directly to the V-Major
- * calls (n_groups = P/2 is the per-GPU scope of the paper).
+ * calls (n_groups = P/2 is the per-GPU scope of the paper).  On one device a
+ * shard is read once and written to both rings' holdings in the same pass.
  * Phase 2 (inter-GPU): one all-to-all per ring t (tile t of every GPU), no
  * traffic between rings: rank 2*g2+t takes its heads from x_p1[t] only.
  * Any (in, out) pair may be NULL/NULL. */

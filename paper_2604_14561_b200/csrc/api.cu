@@ -283,6 +283,7 @@ MoveParams make_pack_params(const uint16_t *const in[3], uint16_t *const out[3],
     p.src_head = D;
     p.dst_tok = D;
     p.dst_head = COMPACT_STRIDE;
+    p.dst2_tok = D;
     p.dst2_head = (long long)S * D;
     p.map = MAP_GATHER;
     p.T = T;
@@ -778,24 +779,24 @@ int cocodiff_tapa_phase1(const uint16_t *q, const uint16_t *k, const uint16_t *v
             if (overlap(in[i], bytes, out[j], 2 * bytes)) return COCODIFF_ALIASING;
             if (i < j && overlap(out[i], 2 * bytes, out[j], 2 * bytes)) return COCODIFF_ALIASING;
         }
-    // The holdings of ring t, p1[t], are a [S][H][D] tensor: tile t keeps its own shard
-    // and receives its partner's.  On one device both are plain row copies.
-    for (int t = 0; t < 2; ++t) {
-        MoveParams p;
-        std::memset(&p, 0, sizeof p);
-        p.n_slots = S;
-        p.H = H;
-        p.D = D;
-        p.src_tok = p.dst_tok = (long long)H * D;
-        p.src_head = p.dst_head = D;
-        p.map = MAP_FULL;
-        p.T = 1;
-        set_extents(p, (long long)E, (long long)E, 0);
-        for (int i = 2; i >= 0; --i)
-            if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i] + (size_t)t * E, nullptr};
-        if (p.njobs == 0) return COCODIFF_OK;
-        CK(launch_move(p, (cudaStream_t)stream));
-    }
+    // The holdings of ring t, p1[t], are a [S][H][D] tensor: tile t keeps its own shard and
+    // receives its partner's.  On one device every shard is read once and written to both
+    // rings' holdings in the same pass.
+    MoveParams p;
+    std::memset(&p, 0, sizeof p);
+    p.n_slots = S;
+    p.H = H;
+    p.D = D;
+    p.src_tok = p.dst_tok = p.dst2_tok = (long long)H * D;
+    p.src_head = p.dst_head = p.dst2_head = D;
+    p.map = MAP_FULL;
+    p.T = 1;
+    set_extents(p, (long long)E, (long long)E, 0);
+    p.dst2_extent = (long long)E;
+    for (int i = 2; i >= 0; --i)
+        if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr, out[i] + E};
+    if (p.njobs == 0) return COCODIFF_OK;
+    CK(launch_selective_move(p, nullptr, (cudaStream_t)stream));
     return COCODIFF_OK;
 }
 

@@ -37,8 +37,9 @@ struct MoveJob {
     const uint16_t *src;
     uint16_t *dst;
     const uint16_t *w;   // RMSNorm weight [D]; nullptr = plain move
-    uint16_t *dst2;      // compaction only: the row is also written to its slot of the cached
-                         // head-parallel tensor [H][S][D] (gather and scatter in one pass); or nullptr
+    uint16_t *dst2;      // a second destination of the same row, or nullptr: its slot of the cached
+                         // head-parallel tensor [H][S][D] (gather and scatter in one pass), or the
+                         // second ring's copy in phase 1 of the two-phase exchange
 };
 
 // One launch moves up to three tensors (jobs) of identical geometry.  Strides
@@ -52,7 +53,7 @@ struct MoveParams {
     int n_slots;            // token slots covered by the grid (capacity)
     int H, D;
     long long src_tok, src_head, dst_tok, dst_head;
-    long long dst2_head;    // head stride of job.dst2 (its token stride is D)
+    long long dst2_tok, dst2_head;  // strides of job.dst2
     const float *cs;        // [S][D/2][2] or nullptr
     float eps;
     const int32_t *idx;     // active units (MAP_GATHER / MAP_SCATTER)

@@ -67,10 +67,10 @@ __device__ __forceinline__ void heads_loop(int &h, const int h_hi, F &&body) {
 // the lanes beyond the row neither load nor store (they add zero to the row's
 // sum of squares).  KIND: what the launch contains; UN / UP = heads in flight per
 // thread on the norm path / the plain path.  TOK = THREADS / LPR token slots per
-// tile.  DUAL: a job may name a second destination (job.dst2), the row's slot
-// in the cached head-parallel tensor, written in the same pass as the compact
-// buffer.  idx_list (shared or global memory) and n_valid (active token slots)
-// are resolved by the calling kernel.
+// tile.  DUAL: a job may name a second destination (job.dst2) that is written
+// in the same pass - the row's slot in the cached head-parallel tensor beside
+// the compact buffer, or the second copy of a shard.  idx_list (shared or global
+// memory) and n_valid (active token slots) are resolved by the calling kernel.
 template <int LPR, bool PAD, int KIND, int UN, int UP, int THREADS, bool DUAL>
 __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b, const int32_t *idx_list,
                                            const int n_valid) {
@@ -136,10 +136,10 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
     (void)dst2_ok;
     const uint4 *sp = reinterpret_cast<const uint4 *>(job.src + s * p.src_tok) + lr + h_lo * sh;
     uint4 *dp = reinterpret_cast<uint4 *>(job.dst + d * p.dst_tok) + lr + h_lo * dh;
-    // second destination: [H][S][D], token stride D
+    // second destination, with strides of its own
     const bool dual = DUAL && job.dst2 != nullptr;
     const long long dh2 = DUAL ? p.dst2_head / 8 : 0;
-    uint4 *dp2 = DUAL ? reinterpret_cast<uint4 *>(job.dst2 + (dual ? d2 * D : 0)) + lr + h_lo * dh2 : nullptr;
+    uint4 *dp2 = DUAL ? reinterpret_cast<uint4 *>(job.dst2 + (dual ? d2 * p.dst2_tok : 0)) + lr + h_lo * dh2 : nullptr;
 
     if (KIND == KIND_PLAIN || (KIND == KIND_MIXED && job.w == nullptr)) {
         if (!valid || !lane_on) return;
