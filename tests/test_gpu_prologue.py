@@ -227,3 +227,57 @@ def test_exchange_and_norm_beyond_2_31_elements():
         assert torch.all((rms - 1.0).abs() < 2.0 ** -8), lo
     # and the normalised rows are the right rows: same signs as the input rows they came from
     assert torch.equal((y.view(S * H, D)[-4096:] < 0), (x.view(S * H, D)[-4096:] < 0))
+
+
+def test_two_host_threads_call_the_library_at_once():
+    """The library keeps no shared mutable state beyond guarded per-device caches and
+    per-thread events: two host threads, each with its own streams and buffers, issue
+    V-first prologues and selective steps concurrently and both get the oracle's results."""
+    import threading
+    cfg = synth.config("tiny")
+    cfg.update(T=16, r=0.5)
+    L = synth.make_layer(cfg)
+    P, S, H, D, T = cfg["P"], cfg["S"], cfg["H"], cfg["D"], cfg["T"]
+    E, n = S * H * D, S // T
+    cs_ref = oracle.rope_table_2d(L["pos"], D, cfg["theta"])
+    want = oracle.prologue(L["q"], L["k"], L["v"], L["wq"], L["wk"], cfg["eps"], cs_ref, P)
+    prev = synth.normal_bf16(3, "prev", E).reshape(S, H, D)
+    m_ref = oracle.vmajor_metric(prev, L["v"], P, T)
+    mask_ref, idx_ref, na_ref = oracle.vmajor_select(m_ref, 1, cfg["r"])
+    errors = []
+
+    def worker(seed):
+        try:
+            torch.cuda.set_device(0)
+            q, k, v, p_v = dev(L["q"]), dev(L["k"]), dev(L["v"]), dev(prev)
+            wq, wk = dev(L["wq"]), dev(L["wk"])
+            cs = rope_table(L["pos"], D, cfg["theta"])
+            out = [torch.zeros(E, dtype=torch.int16, device="cuda") for _ in range(3)]
+            comp = [torch.zeros(E, dtype=torch.int16, device="cuda") for _ in range(3)]
+            metric = torch.zeros(n, dtype=torch.int64, device="cuda")
+            mask = torch.zeros(n, dtype=torch.uint8, device="cuda")
+            idx = torch.zeros(n, dtype=torch.int32, device="cuda")
+            na = torch.zeros(1, dtype=torch.int32, device="cuda")
+            ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
+            ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+            sq, sv = torch.cuda.Stream(), torch.cuda.Stream()
+            for _ in range(200):
+                binding.prologue(q, k, v, *out, wq, wk, cfg["eps"], cs, P, S, H, D, order=binding.V_FIRST,
+                                 stream_qk=sq, stream_v=sv)
+                binding.selective_prologue(p_v, q, k, v, wq, wk, cfg["eps"], cs, P, S, H, D, T, cfg["r"], 1, metric, mask,
+                                           idx, na, *comp, None, None, None, ws, ws_bytes, order=binding.V_FIRST,
+                                           stream_qk=sq, stream_v=sv)
+            sq.synchronize()
+            assert np.array_equal(u16(out[2]).reshape(H, S, D), want[2])
+            assert (u16(out[0]).reshape(H, S, D) != want[0]).mean() < 0.01
+            assert int(na.item()) == na_ref and np.array_equal(idx.cpu().numpy()[:na_ref], idx_ref)
+            assert np.array_equal(mask.cpu().numpy(), mask_ref)
+        except Exception as exc:      # reported by the main thread
+            errors.append((seed, repr(exc)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
