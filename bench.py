@@ -450,10 +450,19 @@ def run_ours(args):
         qk_ms = time_loop(torch, qk_only, sq, args.steps)
         qk_bytes = step_bytes * 2 // 3
         achieved = qk_bytes / (qk_ms * 1e-3) / 1e9
+
+        # context: the library's plain device copy of the same two tensors in the same back-to-back loop
+        def torch_copy():
+            with torch.cuda.stream(sq):
+                qh.copy_(q.reshape(-1))
+                kh.copy_(k.reshape(-1))
+        copy_ms = time_loop(torch, torch_copy, sq, args.steps)
         roofline = {"bound": "hbm", "kernel": "move_rows_kernel<LPR=16, KIND_NORM> (Q and K: RMSNorm + RoPE + exchange, one launch)",
                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                     "frac": achieved / peak, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                     "us_per_launch": 1e3 * qk_ms, "algorithmic_bytes_per_launch": qk_bytes,
+                    "same_loop_torch_copy_of_the_same_bytes": {"us": 1e3 * copy_ms, "gbs": qk_bytes / (copy_ms * 1e-3) / 1e9,
+                                                                "note": "two tensor.copy_ calls (no norm, no rotation, no permutation) timed like the kernel"},
                     "traffic": read_traffic_note(),
                     "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel on this "
                                       "workload, read from profiles/move_rows_kernel_qwen2304.md (not measured in this run)"}
