@@ -16,6 +16,9 @@ Everything is numpy on the host; bf16 tensors are uint16 bit patterns.
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 
 _GOLDEN = np.uint64(0x9E3779B97F4A7C15)
@@ -52,21 +55,31 @@ def random_bits(key: np.uint64, start: int, n: int) -> np.ndarray:
         return _mix64(key + ctr * _GOLDEN)
 
 
+def _normal_chunk(key, s0: int, m: int, mean: float, std: float, out: np.ndarray) -> None:
+    bits = random_bits(key, s0, m)
+    u1 = ((bits >> np.uint64(32)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
+    u2 = ((bits & np.uint64(0xFFFFFFFF)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
+    z = np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
+    out[s0:s0 + m] = (mean + std * z).astype(np.float32)
+
+
 def normal_f32(seed: int, stream: str | int, n: int, mean: float = 0.0,
                std: float = 1.0) -> np.ndarray:
     """n draws of N(mean, std) as float32 (Box-Muller on one 64-bit draw each).
 
-    The value at index i depends only on (seed, stream, i).
+    The value at index i depends only on (seed, stream, i); large requests are
+    filled chunk by chunk on a few host threads (numpy releases the interpreter
+    lock inside its loops), which changes no value.
     """
     key = stream_key(seed, stream)
     out = np.empty(n, dtype=np.float32)
-    for s0 in range(0, n, _CHUNK):
-        m = min(_CHUNK, n - s0)
-        bits = random_bits(key, s0, m)
-        u1 = ((bits >> np.uint64(32)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
-        u2 = ((bits & np.uint64(0xFFFFFFFF)).astype(np.float64) + 0.5) * (1.0 / 4294967296.0)
-        z = np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
-        out[s0:s0 + m] = (mean + std * z).astype(np.float32)
+    chunks = [(s0, min(_CHUNK, n - s0)) for s0 in range(0, n, _CHUNK)]
+    if len(chunks) <= 1:
+        for s0, m in chunks:
+            _normal_chunk(key, s0, m, mean, std, out)
+        return out
+    with ThreadPoolExecutor(max_workers=min(8, len(chunks), os.cpu_count() or 1)) as pool:
+        list(pool.map(lambda c: _normal_chunk(key, c[0], c[1], mean, std, out), chunks))
     return out
 
 
