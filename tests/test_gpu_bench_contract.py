@@ -31,6 +31,7 @@ def test_bench_line_has_every_contract_key():
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert r["traffic"] is None or r["traffic"] > 0.5 * r["algorithmic_bytes_per_launch"]
+    assert r["same_loop_torch_copy_of_the_same_bytes"]["us"] > 0.5 * r["us_per_launch"]
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and "sample" in c
     assert c["all_cores"]["cores"] == len(os.sched_getaffinity(0)) and c["all_cores"]["value"] > 0
@@ -56,3 +57,6 @@ def test_bench_line_has_every_contract_key():
     assert all(row["n_active"] == 29 for row in sel["per_step"]) and sel["n_units"] == 144
     assert sel["algorithmic_bytes"] == 250085376
     assert 0 < pc["launch_floor"]["us"] < pc["tiny"]["lump"]["us_cold_l2"] + 2.0
+    assert pc["sd3"]["lump"]["back_to_back_rotating_buffers"]["exceeds_4x_l2"] is True
+    assert sel["back_to_back_rotating_buffers"]["us_per_step"] > 20.0
+    assert set(c["other_workloads_ms_per_layer"]) == {"tiny", "sd3", "qwen768", "temporal"}
