@@ -85,6 +85,24 @@ SHAPES = [  # P, S, H, D, T, r, n_groups
 ]
 
 
+def _random_shapes(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(count):
+        P = int(rng.choice([1, 2, 3, 4, 6]))
+        H = P * int(rng.integers(1, 4))
+        D = int(rng.choice([8, 24, 32, 56, 64, 104, 128, 192, 256]))
+        T = int(rng.choice([1, 2, 3, 7, 16, 40]))
+        S = P * T * int(rng.integers(1, 60 if T < 16 else 8))
+        n = S // T
+        groups = int(rng.choice([g for g in (1, 2, P, n) if n % g == 0]))
+        out.append((P, S, H, D, T, float(rng.choice([0.0, 0.3, 0.8, 1.0])), groups))
+    return out
+
+
+SHAPES += _random_shapes(8, seed=5)
+
+
 @pytest.mark.parametrize("shape", SHAPES, ids=[str(s[:5]) for s in SHAPES])
 def test_no_access_leaves_its_buffer(shape):
     debug = build.build(debug_bounds=True)
