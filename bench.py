@@ -404,7 +404,9 @@ def run_ours(args):
         stop.record(sq)
         barrier()
         rep_ms.append(max_over_ranks(start.elapsed_time(stop), world, "cuda") / rep_steps)
+    graph_ms = time_graph_loop(torch, lambda: step(binding.V_FIRST), sq, 10, replays=max(2, rep_steps // 10)) if (world == 1 and not args.only_main) else None
     repeats = {"n": 5, "steps_each": rep_steps, "us_per_layer_median": 1e3 * statistics.median(rep_ms),
+               "us_per_layer_as_one_cuda_graph_of_10_steps": None if graph_ms is None else 1e3 * graph_ms,
                "us_per_layer_min": 1e3 * min(rep_ms), "us_per_layer_max": 1e3 * max(rep_ms),
                "gbs_median": aggregate_gbs(step_bytes, world, statistics.median(rep_ms))}
 
