@@ -422,6 +422,15 @@ def run_ours(args):
             orders[name] = {"us_median": 1e3 * statistics.median(ms), "us_min": 1e3 * min(ms),
                             "gbs_median": step_bytes / (statistics.median(ms) * 1e-3) / 1e9,
                             "launches_per_step": 2 if order == binding.V_FIRST else 1}
+
+        def one_stream():
+            binding.prologue(q, k, v, qh, kh, vh, wq, wk, cfg["eps"], cs, P, S, H, D, order=binding.V_FIRST,
+                             stream_qk=sq, stream_v=sq)
+        ms1 = [time_loop(torch, one_stream, sq, rep_steps) for _ in range(5)]
+        orders["v_first_one_stream"] = {"us_back_to_back_median": 1e3 * statistics.median(ms1), "us_back_to_back_min": 1e3 * min(ms1),
+                                        "gbs_median": step_bytes / (statistics.median(ms1) * 1e-3) / 1e9, "launches_per_step": 2,
+                                        "note": "V's launch, then Q/K's with a programmatic dependent launch (no events); "
+                                                "timed like `repeats`"}
         # V-first evidence: V's exchange and the Q/K launch issued as two calls with their own events
         ev = {n: torch.cuda.Event(enable_timing=True) for n in ("v0", "v1", "qk0", "qk1")}
         timeline = []

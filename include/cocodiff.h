@@ -55,8 +55,11 @@ typedef enum {
 
 /* Order of issue of the three exchanges (Section III-C, "V-First Scheduling").
  * LUMP: Q, K and V leave together in one launch on stream_qk (the flat order).
- * V_FIRST: V's exchange is launched first, on stream_v, and runs beside the
- * norm + RoPE + exchange of Q and K on stream_qk.  Results are identical. */
+ * V_FIRST: V's exchange is launched first.  With two streams it runs on stream_v
+ * beside the norm + RoPE + exchange of Q and K on stream_qk.  With stream_v ==
+ * stream_qk the two launches share the stream and are chained with a programmatic
+ * dependent launch: Q/K's grid starts while V's last blocks drain and completes
+ * after it.  Results are identical in every case. */
 typedef enum { COCODIFF_LUMP = 0, COCODIFF_V_FIRST = 1 } cocodiff_order;
 
 const char *cocodiff_status_string(int status);

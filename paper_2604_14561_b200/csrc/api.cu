@@ -130,6 +130,21 @@ int exchange(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *
     base.cs = cs;
     base.eps = eps;
     const bool two_streams = order == COCODIFF_V_FIRST && sv != sq && v != nullptr && (q || k);
+    if (order == COCODIFF_V_FIRST && sv == sq && v != nullptr && (q || k)) {
+        // V first on one stream: V's launch, then Q/K's launch with the programmatic attribute.
+        // Q/K's grid does not read V's output, so it starts while V's last blocks drain, and
+        // waits for V's grid only before it completes (the stream's order of completion holds).
+        MoveParams pv = base;
+        pv.job[pv.njobs++] = MoveJob{v, vh, nullptr, nullptr};
+        pv.pdl = PDL_TRIGGER;
+        MoveParams pqk = base;
+        if (q) pqk.job[pqk.njobs++] = MoveJob{q, qh, wq, nullptr};
+        if (k) pqk.job[pqk.njobs++] = MoveJob{k, kh, wk, nullptr};
+        pqk.pdl = PDL_LAUNCH_ATTR | PDL_WAIT_AT_END;
+        CK(launch_move(pv, sq));
+        CK(launch_move(pqk, sq));
+        return COCODIFF_OK;
+    }
     if (order == COCODIFF_LUMP || !two_streams) {
         // one launch; V's blocks come first in the grid
         MoveParams p = base;

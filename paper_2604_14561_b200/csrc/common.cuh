@@ -20,6 +20,7 @@ enum TokenMap : int {
 enum PdlFlags : int {
     PDL_WAIT_AT_START = 1,   // the kernel consumes its predecessor's results
     PDL_TRIGGER = 2,         // let the successor start as soon as every block of this grid runs
+    PDL_WAIT_AT_END = 4,     // independent of the predecessor, but must not complete before it
     PDL_LAUNCH_ATTR = 8      // host side: launch with programmatic stream serialization
 };
 

@@ -44,6 +44,9 @@ __global__ void __launch_bounds__(kThreads, kMinBlocks) move_rows_kernel(const _
         if (n_valid < 0) n_valid = 0;
     }
     move_block<LPR, PAD, KIND, UN, UP, kThreads, false>(p, blockIdx.x, p.idx, n_valid);
+    // A grid that started beside its predecessor without consuming its results still has to
+    // complete after it: whoever waits for this grid then also has the predecessor's output.
+    if (p.pdl & PDL_WAIT_AT_END) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 template <int LPR, bool PAD>

@@ -93,9 +93,9 @@ def test_prologue_parity_full_size_21k_tokens():
     cfg = synth.config("qwen2304")
     L = synth.make_layer(cfg)
     a, _ = _check_prologue(L, cfg, order=binding.V_FIRST, report="qwen2304")
-    b = run_prologue(L, cfg, order=binding.LUMP)
-    for x, y in zip(a, b):
-        assert np.array_equal(x, y), "the order of issue must not change any value"
+    for b in (run_prologue(L, cfg, order=binding.LUMP), run_prologue(L, cfg, order=binding.V_FIRST, two_streams=False)):
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y), "the order of issue must not change any value"
 
 
 @pytest.mark.parametrize("P,S,H,D", [(1, 37, 1, 32), (1, 5, 3, 64), (3, 33, 3, 128), (2, 1002, 6, 256),
@@ -107,6 +107,7 @@ def test_prologue_ragged_and_degenerate_shapes(P, S, H, D):
     L, cfg = _layer(P, S, H, D, seed=100 + S)
     _check_prologue(L, cfg, order=binding.V_FIRST)
     _check_prologue(L, cfg, order=binding.LUMP, two_streams=False)
+    _check_prologue(L, cfg, order=binding.V_FIRST, two_streams=False)      # V first on one stream
 
 
 def test_empty_sequence_is_a_no_op():
