@@ -719,24 +719,6 @@ def temporal_rows(torch, binding, args):
         "launches_per_step": {"lump": 2, "v_first": 3},
         "kernel_break_out": "per-kernel durations of these same launches: profiles/vmajor_selective_step_temporal.md (ncu)",
         "api": "cocodiff_selective_prologue"}
-    # Selective steps back to back on two rotating buffer sets (1.1 GB together, more than four times
-    # the L2), captured as one CUDA graph: no event, flush or host work between the steps.
-    sets = [(steps[t - 1]["v"], steps[t], [new() for _ in range(3)], [new() for _ in range(3)]) for t in (1, 2)]
-    calls = [0]
-
-    def rotating():
-        prev, x, cmp_, cch = sets[calls[0] % 2]
-        calls[0] += 1
-        binding.selective_prologue(prev, x["q"], x["k"], x["v"], wq, wk, cfg["eps"], cs, P, S, H, D, T, r, n_groups,
-                                   metric, mask, idx, na, *cmp_, *cch, ws, binding.vmajor_workspace_bytes(P, S, H, D, T),
-                                   order=binding.LUMP, stream_qk=sq, stream_v=sq)
-    ms = time_graph_loop(torch, rotating, sq, 4, replays=10)
-    if ms is not None:
-        out["steps_1_to_7_selective"]["back_to_back_rotating_buffers"] = {
-            "us_per_step": 1e3 * ms, "gbs_on_algorithmic_bytes": b_alg / (ms * 1e-3) / 1e9,
-            "gbs_on_bytes_moved": b_moved / (ms * 1e-3) / 1e9, "frac_of_measured_copy_peak_on_bytes_moved": b_moved / (ms * 1e-3) / 1e9 / peak,
-            "how": "one CUDA graph of 4 consecutive steps alternating between two buffer sets, replayed 10 times (median of 5)"}
-    del sets
     # the metric pass and its selection alone (no compaction follows, so the selection is a launch of
     # its own), and - for context - a library read-only reduction over the same two tensors
     def metric_alone():
@@ -765,6 +747,34 @@ def temporal_rows(torch, binding, args):
             "us_cold_l2": t1, "n_units": S, "n_active": n_act1, "algorithmic_bytes": b1,
             "gbs_on_algorithmic_bytes": b1 / (t1 * 1e-6) / 1e9, "ratio_to_64_token_tiles": t1 / per_step[0]["us_lump"],
             "launches_per_step": 3}
+    # Selective steps back to back on two rotating buffer sets (1.1 GB together, more than four times
+    # the L2), captured as one CUDA graph: no event, flush or host work between the steps.  This is
+    # also the only figure here that the 2 µs grain of the event stamps does not touch.
+    sets = [(steps[t - 1]["v"], steps[t], [new() for _ in range(3)], [new() for _ in range(3)]) for t in (1, 2)]
+
+    def rotating_loop(T_, groups):
+        calls = [0]
+
+        def rotating():
+            prev, x, cmp_, cch = sets[calls[0] % 2]
+            calls[0] += 1
+            binding.selective_prologue(prev, x["q"], x["k"], x["v"], wq, wk, cfg["eps"], cs, P, S, H, D, T_, r, groups,
+                                       metric, mask, idx, na, *cmp_, *cch, ws, binding.vmajor_workspace_bytes(P, S, H, D, T_),
+                                       order=binding.LUMP, stream_qk=sq, stream_v=sq)
+        return time_graph_loop(torch, rotating, sq, 4, replays=10)
+    how = "one CUDA graph of 4 consecutive steps alternating between two buffer sets, replayed 10 times (median of 5)"
+    ms = rotating_loop(T, n_groups)
+    if ms is not None:
+        out["steps_1_to_7_selective"]["back_to_back_rotating_buffers"] = {
+            "us_per_step": 1e3 * ms, "gbs_on_algorithmic_bytes": b_alg / (ms * 1e-3) / 1e9,
+            "gbs_on_bytes_moved": b_moved / (ms * 1e-3) / 1e9, "frac_of_measured_copy_peak_on_bytes_moved": b_moved / (ms * 1e-3) / 1e9 / peak,
+            "how": how}
+        for groups in (1, P):
+            ms1 = rotating_loop(1, groups)
+            if ms1 is not None:
+                out[f"step_1_per_token_units_groups{groups}"]["back_to_back_rotating_buffers"] = {
+                    "us_per_step": 1e3 * ms1, "ratio_to_64_token_tiles": ms1 / ms, "how": how}
+    del sets
     return out
 
 

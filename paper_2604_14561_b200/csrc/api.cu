@@ -330,6 +330,7 @@ int enqueue_select_and_pack(const SelectionPlan &pl, const uint16_t *const in[3]
                             uint16_t *const cache[3], const uint16_t *wq, const uint16_t *wk, float eps,
                             const float *cs, int slots, int S, int H, int D, int T, cudaStream_t st) {
     MoveParams p = make_pack_params(in, out, cache, wq, wk, eps, cs, pl.sp.idx, pl.sp.n_active, slots, S, H, D, T);
+    p.slots_exact = 1;  // slots = (n - n_groups * floor(r * g)) * T, what the selection will publish
     // the consuming kernel selects for itself when it has few units to rank and at least one block
     const bool consume = p.njobs > 0 && pl.in_consumer && slots > 0;
     MetricParams mp = pl.mp;
@@ -731,6 +732,7 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
     uint16_t *cache_qk[3] = {q_cache, k_cache, nullptr};
     MoveParams p = make_pack_params(in_qk, out_qk, do_unpack ? cache_qk : nullptr, wq, wk, eps, cs, idx, n_active, slots, S,
                                     H, D, T);
+    p.slots_exact = 1;
     CK(launch_selective_move(p, nullptr, sq));
     return COCODIFF_OK;
 }

@@ -52,6 +52,7 @@ struct MoveParams {
     MoveJob job[3];
     int njobs;
     int n_slots;            // token slots covered by the grid (capacity)
+    int slots_exact;        // n_slots IS n_active * T (the host derived it from the rule): n_active is not read
     int H, D;
     long long src_tok, src_head, dst_tok, dst_head;
     long long dst2_tok, dst2_head;  // strides of job.dst2

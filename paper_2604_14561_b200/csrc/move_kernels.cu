@@ -60,8 +60,8 @@ selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constan
     if (select_here) {
         nv = (long long)vmajor::select_small<kThreads>(sel, 0, sel.n, sm, blockIdx.x == 0) * p.T;
         list = sm.idx;
-    } else if (p.map == MAP_FULL) {
-        nv = p.n_slots;  // every slot moves (a plain move with two destinations)
+    } else if (p.map == MAP_FULL || p.slots_exact) {
+        nv = p.n_slots;  // every slot moves: a plain move, or a grid sized from the rule's own count
     } else {
         nv = (long long)__ldcg(p.n_active) * p.T;
     }

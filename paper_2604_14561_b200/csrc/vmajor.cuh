@@ -387,6 +387,7 @@ __device__ void emit_selection(const SelectParams &p, int grp, const unsigned lo
     __syncthreads();
 }
 
+// dyn: the histogram words are ZERO on entry when n_cached != 0 and g <= 65535.
 template <int BLOCK>
 __device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm, unsigned *dyn, const int mb) {
     const int tid = threadIdx.x, lane = tid & 31;
@@ -409,14 +410,13 @@ __device__ void select_group_large(const SelectParams &p, int grp, LargeSel &sm,
         int *warp_hist = reinterpret_cast<int *>(dyn);
         const int k = n_cached - 1;
         if (keyed) {
-            // one pass over the metrics (sixteen loads in flight per thread, the first batch
-            // issued before the histogram is cleared): keys and their histogram
+            // one pass over the metrics (sixteen loads in flight per thread): keys and their
+            // histogram (dyn[0 .. hist_words) is zero on entry)
             constexpr int UL = 16;
             unsigned long long v[UL];
 #pragma unroll
             for (int u = 0; u < UL; ++u) v[u] = tid + u * BLOCK < g ? __ldcg(vals + tid + u * BLOCK) : 0ull;
-            for (int i = tid; i < hist_words; i += BLOCK) dyn[i] = 0;
-            __syncthreads();
+            __syncthreads();  // the histogram was cleared by the caller, before it waited for the metrics
             for (int e0 = tid; e0 < g; e0 += UL * BLOCK) {
                 if (e0 != tid) {
 #pragma unroll

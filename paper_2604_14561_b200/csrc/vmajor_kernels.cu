@@ -35,6 +35,9 @@ vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int mb,
     __shared__ LargeSel sm;
     extern __shared__ __align__(16) unsigned dyn_words[];
     if (pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // the histogram is cleared while the kernel that produces the metrics still drains
+    if (p.n_cached != 0 && p.g <= 65535)
+        for (int i = threadIdx.x; i < (int)(large_hist_bytes(mb) / 4); i += kLargeBlock) dyn_words[i] = 0;
     if (pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
     select_group_large<kLargeBlock>(p, blockIdx.x, sm, dyn_words, mb);
 }
