@@ -680,10 +680,10 @@ def temporal_rows(torch, binding, args):
         binding.prologue(x["q"], x["k"], x["v"], *cache, wq, wk, cfg["eps"], cs, P, S, H, D, order=order,
                          stream_qk=sq, stream_v=sv)
 
-    def selective(t, order, T_=T, groups=n_groups):
+    def selective(t, order, T_=T, groups=n_groups, direct=False):
         x, prev = steps[t], steps[t - 1]["v"]
         binding.selective_prologue(prev, x["q"], x["k"], x["v"], wq, wk, cfg["eps"], cs, P, S, H, D, T_, r, groups,
-                                   metric, mask, idx, na, *comp, *cache,
+                                   metric, mask, idx, na, *([None] * 3 if direct else comp), *cache,
                                    ws, binding.vmajor_workspace_bytes(P, S, H, D, T_), order=order,
                                    stream_qk=sq, stream_v=sv if order == binding.V_FIRST else sq)
     out = {"workload": "temporal: P=24, S=9216, H=24, D=128, T=64, r=0.8, one global group; 8 steps of the data law",
@@ -719,6 +719,17 @@ def temporal_rows(torch, binding, args):
         "launches_per_step": {"lump": 2, "v_first": 3},
         "kernel_break_out": "per-kernel durations of these same launches: profiles/vmajor_selective_step_temporal.md (ncu)",
         "api": "cocodiff_selective_prologue"}
+    # Direct delivery: no compact buffers, the active rows are stored straight to their slots of the
+    # cached tensors (what a sender does over NVLink peer memory); one read and one write per active row.
+    td = [1e3 * statistics.mean(time_steps(torch, lambda: selective(t, binding.LUMP, direct=True), sq, iters, 3, flush=flush))
+          for t in range(1, cfg["steps"])]
+    b_direct = 2 * E * 2 + 6 * n_act * tile
+    out["steps_1_to_7_selective_direct_delivery"] = {
+        "us_per_step": td, "us_mean": statistics.mean(td), "algorithmic_bytes": b_direct,
+        "gbs_on_algorithmic_bytes": b_direct / (statistics.mean(td) * 1e-6) / 1e9,
+        "frac_of_measured_copy_peak": b_direct / (statistics.mean(td) * 1e-6) / 1e9 / peak,
+        "note": "cocodiff_selective_prologue with the three compact buffers NULL: metric pass (2 tensors read) + "
+                "active rows of Q, K, V read once and written once; the caches receive the same bits as above"}
     # the metric pass and its selection alone (no compaction follows, so the selection is a launch of
     # its own), and - for context - a library read-only reduction over the same two tensors
     def metric_alone():
@@ -752,14 +763,15 @@ def temporal_rows(torch, binding, args):
     # also the only figure here that the 2 µs grain of the event stamps does not touch.
     sets = [(steps[t - 1]["v"], steps[t], [new() for _ in range(3)], [new() for _ in range(3)]) for t in (1, 2)]
 
-    def rotating_loop(T_, groups):
+    def rotating_loop(T_, groups, direct=False):
         calls = [0]
 
         def rotating():
             prev, x, cmp_, cch = sets[calls[0] % 2]
             calls[0] += 1
             binding.selective_prologue(prev, x["q"], x["k"], x["v"], wq, wk, cfg["eps"], cs, P, S, H, D, T_, r, groups,
-                                       metric, mask, idx, na, *cmp_, *cch, ws, binding.vmajor_workspace_bytes(P, S, H, D, T_),
+                                       metric, mask, idx, na, *([None] * 3 if direct else cmp_), *cch, ws,
+                                       binding.vmajor_workspace_bytes(P, S, H, D, T_),
                                        order=binding.LUMP, stream_qk=sq, stream_v=sq)
         return time_graph_loop(torch, rotating, sq, 4, replays=10)
     how = "one CUDA graph of 4 consecutive steps alternating between two buffer sets, replayed 10 times (median of 5)"
@@ -769,6 +781,11 @@ def temporal_rows(torch, binding, args):
             "us_per_step": 1e3 * ms, "gbs_on_algorithmic_bytes": b_alg / (ms * 1e-3) / 1e9,
             "gbs_on_bytes_moved": b_moved / (ms * 1e-3) / 1e9, "frac_of_measured_copy_peak_on_bytes_moved": b_moved / (ms * 1e-3) / 1e9 / peak,
             "how": how}
+        msd = rotating_loop(T, n_groups, direct=True)
+        if msd is not None:
+            out["steps_1_to_7_selective_direct_delivery"]["back_to_back_rotating_buffers"] = {
+                "us_per_step": 1e3 * msd, "gbs_on_algorithmic_bytes": b_direct / (msd * 1e-3) / 1e9,
+                "frac_of_measured_copy_peak": b_direct / (msd * 1e-3) / 1e9 / peak, "how": how}
         for groups in (1, P):
             ms1 = rotating_loop(1, groups)
             if ms1 is not None:
@@ -828,24 +845,30 @@ def next_rows(torch, binding, args, rows=("inverse", "tapa", "schedule", "moves"
     na = torch.zeros(1, dtype=torch.int32, device="cuda")
     if "schedule" in rows:
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(total + 1)]
-        for rep in range(2):                 # first pass warms up
-            sent = []
-            torch.cuda.synchronize()
-            ev[0].record(sq)
-            for step_i in range(total):
-                _, s_el = binding.layer_step(step_i, total, warmup, interval, v, q, k, v, wq, wk,
-                                             cfg["eps"], cs, P, S, H, D, T, 1, metric, mask, idx, na, comp[0], comp[1],
-                                             comp[2], qh, kh, vh, ws, ws_bytes, order=binding.LUMP, stream_qk=sq, stream_v=sq)
-                sent.append(s_el)
-                ev[step_i + 1].record(sq)
-            torch.cuda.synchronize()
-        per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(total)]
         full = [binding.cache_schedule(i, total, warmup, interval)[0] for i in range(total)]
-        out["schedule_50_steps"] = {
-            "total_us": 1e3 * sum(per_step), "always_full_us_estimate": 1e3 * total * statistics.mean(t for t, f in zip(per_step, full) if f),
-            "full_steps": sum(full), "us_full_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if f),
-            "us_selective_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if not f),
-            "exchanged_fraction_of_always_full": sum(sent) / (total * 3 * E), "l2": "warm (steps back to back)"}
+        for name, bufs in (("schedule_50_steps", comp), ("schedule_50_steps_direct_delivery", [None] * 3)):
+            for rep in range(2):                 # first pass warms up
+                sent = []
+                torch.cuda.synchronize()
+                ev[0].record(sq)
+                for step_i in range(total):
+                    _, s_el = binding.layer_step(step_i, total, warmup, interval, v, q, k, v, wq, wk,
+                                                 cfg["eps"], cs, P, S, H, D, T, 1, metric, mask, idx, na, *bufs,
+                                                 qh, kh, vh, ws, ws_bytes, order=binding.LUMP, stream_qk=sq, stream_v=sq)
+                    sent.append(s_el)
+                    ev[step_i + 1].record(sq)
+                torch.cuda.synchronize()
+            per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(total)]
+            out[name] = {
+                "total_us": 1e3 * sum(per_step),
+                "always_full_us_estimate": 1e3 * total * statistics.mean(t for t, f in zip(per_step, full) if f),
+                "full_steps": sum(full), "us_full_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if f),
+                "us_selective_step_mean": 1e3 * statistics.mean(t for t, f in zip(per_step, full) if not f),
+                "exchanged_fraction_of_always_full": sum(sent) / (total * 3 * E), "l2": "warm (steps back to back)"}
+        out["schedule_50_steps"]["note"] = (
+            "on one device a selective step is sender and receiver at once: metric pass + active rows read once and "
+            "written twice (send buffer and cache), so it moves fewer bytes than a full step only for r > 0.56; "
+            "with direct delivery (no send buffer) for r > 0.33")
     if "moves" not in rows:
         return out
     # the stand-alone compaction and the receiver-only scatter of 29 of 144 units (the selective step

@@ -199,7 +199,13 @@ int cocodiff_unpack_qkv(const uint16_t *q_compact, const uint16_t *k_compact, co
  * compactions in one launch.  Consecutive kernels of a stream are chained with
  * programmatic dependent launches.  Stream semantics as for
  * cocodiff_ulysses_a2a; outputs and workspace as for
- * cocodiff_vmajor_select_compact.  The caches are all given or all NULL. */
+ * cocodiff_vmajor_select_compact.  The caches are all given or all NULL.
+ * Direct delivery: with the caches given, the three compact buffers may all be
+ * NULL; the active rows are then stored straight to their slots of the cached
+ * HEAD tensors (between NVLink peers: a store into the receiver's memory) and
+ * no send buffer is written.  The caches end up with the same bits either way.
+ * Compact buffers that are given are all given; all NULL without the caches is
+ * INVALID_ARG. */
 int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const uint16_t *k, const uint16_t *v,
                                 const uint16_t *wq, const uint16_t *wk, float eps, const float *cs,
                                 int P, int S, int H, int D, int T, double r, int n_groups,
@@ -224,7 +230,7 @@ int cocodiff_cache_schedule(int step, int total_steps, int warmup, int sync_inte
  * cocodiff_prologue straight into the three caches (resetting them to the exact
  * values of this step); a selective step runs cocodiff_selective_prologue with
  * the scheduled r.  All arguments as in those two calls; the caches are
- * required.  sent_elements (HOST pointer, may be NULL) receives the number of
+ * required, the compact buffers may all be NULL (direct delivery).  sent_elements (HOST pointer, may be NULL) receives the number of
  * bf16 elements of Q, K, V that cross the exchange in this step. */
 int cocodiff_layer_step(int step, int total_steps, int warmup, int sync_interval,
                         const uint16_t *prev_v, const uint16_t *q, const uint16_t *k, const uint16_t *v,

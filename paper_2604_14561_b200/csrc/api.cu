@@ -286,9 +286,10 @@ SelectionPlan plan_selection(const uint16_t *prev_v, const uint16_t *cur_v, int 
 
 // Compaction of up to three tensors in one launch; slot order (Q, K, V), V's blocks first.
 // cache[i], when given, also receives the rows (the receiver-side scatter in the same pass).
+// direct: there is no compact buffer; the rows go to their slots of cache[i] only.
 MoveParams make_pack_params(const uint16_t *const in[3], uint16_t *const out[3], uint16_t *const cache[3],
                             const uint16_t *wq, const uint16_t *wk, float eps, const float *cs, const int32_t *idx,
-                            const int32_t *n_active, int slots, int S, int H, int D, int T) {
+                            const int32_t *n_active, int slots, int S, int H, int D, int T, bool direct = false) {
     MoveParams p;
     std::memset(&p, 0, sizeof p);
     p.n_slots = slots;
@@ -309,6 +310,14 @@ MoveParams make_pack_params(const uint16_t *const in[3], uint16_t *const out[3],
     p.eps = eps;
     set_extents(p, (long long)S * H * D, (long long)S * H * D, (long long)S * D);
     p.dst2_extent = (long long)S * H * D;
+    if (direct) {
+        p.map = MAP_ACTIVE;
+        p.dst_head = (long long)S * D;
+        if (in[2]) p.job[p.njobs++] = MoveJob{in[2], cache[2], nullptr, nullptr};
+        if (in[0]) p.job[p.njobs++] = MoveJob{in[0], cache[0], wq, nullptr};
+        if (in[1]) p.job[p.njobs++] = MoveJob{in[1], cache[1], wk, nullptr};
+        return p;
+    }
     if (in[2]) p.job[p.njobs++] = MoveJob{in[2], out[2], nullptr, cache ? cache[2] : nullptr};
     if (in[0]) p.job[p.njobs++] = MoveJob{in[0], out[0], wq, cache ? cache[0] : nullptr};
     if (in[1]) p.job[p.njobs++] = MoveJob{in[1], out[1], wk, cache ? cache[1] : nullptr};
@@ -328,8 +337,10 @@ int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint
 // chained with programmatic dependent launches.
 int enqueue_select_and_pack(const SelectionPlan &pl, const uint16_t *const in[3], uint16_t *const out[3],
                             uint16_t *const cache[3], const uint16_t *wq, const uint16_t *wk, float eps,
-                            const float *cs, int slots, int S, int H, int D, int T, cudaStream_t st) {
-    MoveParams p = make_pack_params(in, out, cache, wq, wk, eps, cs, pl.sp.idx, pl.sp.n_active, slots, S, H, D, T);
+                            const float *cs, int slots, int S, int H, int D, int T, cudaStream_t st,
+                            bool direct = false) {
+    MoveParams p =
+        make_pack_params(in, out, cache, wq, wk, eps, cs, pl.sp.idx, pl.sp.n_active, slots, S, H, D, T, direct);
     p.slots_exact = 1;  // slots = (n - n_groups * floor(r * g)) * T, what the selection will publish
     // the consuming kernel selects for itself when it has few units to rank and at least one block
     const bool consume = p.njobs > 0 && pl.in_consumer && slots > 0;
@@ -679,22 +690,26 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
                           workspace_bytes);
     if (rc) return rc;
     if (order != COCODIFF_LUMP && order != COCODIFF_V_FIRST) return COCODIFF_INVALID_ARG;
-    if (!q || !k || !wq || !wk || !cs || !q_compact || !k_compact || !v_compact || !(eps >= 0.f))
-        return COCODIFF_INVALID_ARG;
+    if (!q || !k || !wq || !wk || !cs || !(eps >= 0.f)) return COCODIFF_INVALID_ARG;
     if (!aligned16(wq) || !aligned16(wk) || !aligned16(cs)) return COCODIFF_MISALIGNED;
     const bool do_unpack = q_cache || k_cache || v_cache;
     if (do_unpack && !(q_cache && k_cache && v_cache)) return COCODIFF_INVALID_ARG;
+    // direct delivery: no compact buffers, the active rows go straight to the caches
+    const bool direct = !q_compact && !k_compact && !v_compact;
+    if (direct ? !do_unpack : !(q_compact && k_compact && v_compact)) return COCODIFF_INVALID_ARG;
     const uint16_t *in[3] = {q, k, v};
     uint16_t *comp[3] = {q_compact, k_compact, v_compact};
-    rc = check_tiles(in, comp, S, H, D, idx, n_active);
-    if (rc) return rc;
     const size_t bytes = (size_t)S * H * D * 2;
-    for (int i = 0; i < 3; ++i)
-        if (overlap(prev_v, bytes, comp[i], bytes)) return COCODIFF_ALIASING;
+    if (!direct) {
+        rc = check_tiles(in, comp, S, H, D, idx, n_active);
+        if (rc) return rc;
+        for (int i = 0; i < 3; ++i)
+            if (overlap(prev_v, bytes, comp[i], bytes)) return COCODIFF_ALIASING;
+    }
     const uint16_t *comp_in[3] = {q_compact, k_compact, v_compact};
     uint16_t *cache[3] = {q_cache, k_cache, v_cache};
     if (do_unpack) {
-        rc = check_tiles(comp_in, cache, S, H, D, idx, n_active);
+        rc = check_tiles(direct ? in : comp_in, cache, S, H, D, idx, n_active);
         if (rc) return rc;
         for (int i = 0; i < 3; ++i)
             for (int j = 0; j < 3; ++j)
@@ -710,7 +725,7 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
     // chained with programmatic dependent launches: each successor becomes resident while
     // its predecessor drains and orders itself with griddepcontrol.wait.
     if (order == COCODIFF_LUMP || sv == sq)
-        return enqueue_select_and_pack(pl, in, comp, scatter, wq, wk, eps, cs, slots, S, H, D, T, sq);
+        return enqueue_select_and_pack(pl, in, comp, scatter, wq, wk, eps, cs, slots, S, H, D, T, sq, direct);
     // V first: metric, selection and V's compaction + scatter on stream_v; Q and K follow on
     // stream_qk once V's part is done and read the list that V's part published.
     ForkJoin *fj = nullptr;
@@ -722,7 +737,7 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
     uint16_t *out_v[3] = {nullptr, nullptr, v_compact};
     uint16_t *cache_v[3] = {nullptr, nullptr, v_cache};
     rc = enqueue_select_and_pack(pl, in_v, out_v, do_unpack ? cache_v : nullptr, nullptr, nullptr, 0.f, nullptr, slots, S, H,
-                                 D, T, sv);
+                                 D, T, sv, direct);
     // whatever happened on stream_v, stream_qk is ordered behind it again
     const int rj = join_streams(fj, sq, sv);
     if (rc) return rc;
@@ -731,7 +746,7 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
     uint16_t *out_qk[3] = {q_compact, k_compact, nullptr};
     uint16_t *cache_qk[3] = {q_cache, k_cache, nullptr};
     MoveParams p = make_pack_params(in_qk, out_qk, do_unpack ? cache_qk : nullptr, wq, wk, eps, cs, idx, n_active, slots, S,
-                                    H, D, T);
+                                    H, D, T, direct);
     p.slots_exact = 1;
     CK(launch_selective_move(p, nullptr, sq));
     return COCODIFF_OK;

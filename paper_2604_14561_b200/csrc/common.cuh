@@ -9,7 +9,8 @@ namespace cocodiff {
 enum TokenMap : int {
     MAP_FULL = 0,     // src token = dst token = o                      (full exchange)
     MAP_GATHER = 1,   // src token = idx[o / T] * T + o % T, dst = o    (compaction)
-    MAP_SCATTER = 2   // src token = o, dst token = idx[o / T] * T + o % T  (reconstruction)
+    MAP_SCATTER = 2,  // src token = o, dst token = idx[o / T] * T + o % T  (reconstruction)
+    MAP_ACTIVE = 3    // src token = dst token = idx[o / T] * T + o % T   (direct delivery: no send buffer)
 };
 
 // Programmatic dependent launch (same-stream overlap of consecutive kernels).

@@ -30,6 +30,8 @@ using namespace rows;
 // 4 blocks per SM (<= 64 registers), evict-first accesses; heads per block and
 // loads in flight per thread depend on what the launch contains.
 constexpr int kThreads = 256, kMinBlocks = 4;
+// heads per item of the selective mover (items of 2 to 24 heads measured: 6 and 12 are the fastest)
+constexpr int kSelHeads = 6;
 
 // Grid: one block per (head range, job, token tile); THREADS x MINB = threads resident per SM.
 template <int LPR, bool PAD, int KIND, int UN, int UP>
@@ -76,7 +78,7 @@ selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constan
     const unsigned groups = (unsigned)p.head_split * (unsigned)p.njobs;   // (head range, tensor) pairs
     for (unsigned item = blockIdx.x; item < tiles * groups; item += gridDim.x) {
         const unsigned grp = item / tiles, tile = item - grp * tiles;
-        move_block<LPR, PAD, KIND_MIXED, 4, 4, kThreads, true>(p, grp * tiles_cap + tile, list, n_valid);
+        move_block<LPR, PAD, KIND_MIXED, 4, 4, kThreads, true, kSelHeads>(p, grp * tiles_cap + tile, list, n_valid);
     }
 }
 
@@ -138,7 +140,7 @@ template <int LPR, bool PAD>
 cudaError_t launch_selective_lpr(MoveParams p, const SelectParams *sel, cudaStream_t stream) {
     static const SelectParams none = {};
     // items of 6 heads: fine enough to balance one resident wave (4 blocks on each SM)
-    const long long items = grid_blocks(p, LPR, 6);
+    const long long items = grid_blocks(p, LPR, kSelHeads);
     if (items > 0xffffffffLL) return cudaErrorInvalidConfiguration;
     const long long wave = (long long)sm_count() * kMinBlocks;
     return launch_grid(selective_move_kernel<LPR, PAD>, items < wave ? items : wave, stream, p.pdl, p, sel ? *sel : none,

@@ -71,7 +71,8 @@ __device__ __forceinline__ void heads_loop(int &h, const int h_hi, F &&body) {
 // in the same pass - the row's slot in the cached head-parallel tensor beside
 // the compact buffer, or the second copy of a shard.  idx_list (shared or global
 // memory) and n_valid (active token slots) are resolved by the calling kernel.
-template <int LPR, bool PAD, int KIND, int UN, int UP, int THREADS, bool DUAL>
+// PF: source rows (heads) requested from the L2 ahead of the block's own loads.
+template <int LPR, bool PAD, int KIND, int UN, int UP, int THREADS, bool DUAL, int PF = 0>
 __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b, const int32_t *idx_list,
                                            const int n_valid) {
     constexpr int TOK = THREADS / LPR;  // token slots per tile
@@ -115,7 +116,8 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
         int unit = idx_list[a];  // a list that was never written must not send accesses out of bounds
         unit = unit < 0 ? 0 : (unit >= p.n_units ? p.n_units - 1 : unit);
         const long long tk = (long long)unit * p.T + (o - a * p.T);
-        if (p.map == MAP_GATHER) s = tk; else d = tk;
+        if (p.map != MAP_SCATTER) s = tk;
+        if (p.map != MAP_GATHER) d = tk;
         d2 = tk;
     }
     // bounds-checked build only: is the 16-byte vector at ptr inside its buffer?
@@ -141,6 +143,15 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
     const long long dh2 = DUAL ? p.dst2_head / 8 : 0;
     uint4 *dp2 = DUAL ? reinterpret_cast<uint4 *>(job.dst2 + (dual ? d2 * p.dst2_tok : 0)) + lr + h_lo * dh2 : nullptr;
 
+    // A block that walks a few items of scattered units meets the memory latency anew at every
+    // item (the list, then the per-token constants, then the rows): the rows of the first PF
+    // heads are asked of the L2 before the constants are loaded.  (Whole-tensor moves and grids
+    // of one item per block hide that latency behind their other work, and measured slower
+    // with the extra requests.)
+    if (PF > 0 && p.map != MAP_FULL && lane_on) {
+        const int np = h_hi - h_lo < PF ? h_hi - h_lo : PF;
+        for (int u = 0; u < np; ++u) asm volatile("prefetch.global.L2 [%0];" ::"l"(sp + u * sh));
+    }
     if (KIND == KIND_PLAIN || (KIND == KIND_MIXED && job.w == nullptr)) {
         if (!valid || !lane_on) return;
         int h = h_lo;

@@ -97,6 +97,28 @@ def test_vmajor_validation():
     assert binding.unpack(comp, None, na, cur, 2, 64, 4, 64, 8, check=False) == -1
 
 
+def test_selective_prologue_validation_of_direct_delivery():
+    """Compact buffers are all given or all NULL, and all NULL only with the caches."""
+    prev, q, k, v = (_addr(i) * 64 for i in range(4))
+    comp = [_addr(4 + i) * 64 for i in range(3)]
+    cache = [_addr(8 + i) * 64 for i in range(3)]
+    m, mask, idx, na, ws, w, cs = (_addr(100 + i) for i in range(7))
+    need = binding.vmajor_workspace_bytes(2, 64, 4, 64, 8)
+
+    def call(comp, cache):
+        return binding.selective_prologue(prev, q, k, v, w, w, 1e-6, cs, 2, 64, 4, 64, 8, 0.5, 1, m, mask, idx, na,
+                                          *comp, *cache, ws, need, check=False)
+    none = [None] * 3
+    assert call(none, none) == -1                              # nowhere to deliver to
+    assert call([comp[0], None, comp[2]], cache) == -1         # half a set of compact buffers
+    assert call([None, None, comp[2]], cache) == -1
+    assert call(comp, [cache[0], None, None]) == -1            # half a set of caches
+    assert call(none, [cache[0], cache[0], cache[2]]) == -6    # two caches on one buffer
+    assert call(none, [q, cache[1], cache[2]]) == -6           # a cache over an input
+    assert call(none, [prev, cache[1], cache[2]]) == -6
+    assert call(none, [cache[0] + 2, cache[1], cache[2]]) == -3
+
+
 def test_static_unit_limit_is_the_headers():
     text = open(os.path.join(ROOT, "include", "cocodiff.h")).read()
     m = re.search(r"#define\s+COCODIFF_STATIC_MAX_UNITS\s+(\d+)", text)

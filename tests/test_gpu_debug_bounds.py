@@ -64,6 +64,12 @@ def _run_everything(P, S, H, D, T, r, n_groups, seed):
     for order, s_v in ((binding.LUMP, sq), (binding.V_FIRST, sv)):
         binding.selective_prologue(prev, x["q"], x["k"], x["v"], wq, wk, 1e-6, cs, P, S, H, D, T, r, n_groups,
                                    metric, mask, idx, na, *comp, *cache, ws, ws_bytes, order=order, stream_qk=sq, stream_v=s_v)
+    direct = [new() for _ in range(3)]      # no compact buffers: straight to the caches
+    for order, s_v in ((binding.LUMP, sq), (binding.V_FIRST, sv)):
+        binding.selective_prologue(prev, x["q"], x["k"], x["v"], wq, wk, 1e-6, cs, P, S, H, D, T, r, n_groups,
+                                   metric, mask, idx, na, None, None, None, *direct, ws, ws_bytes, order=order,
+                                   stream_qk=sq, stream_v=s_v)
+    outs += direct
     vc = new()
     binding.vmajor_select_compact(prev, x["v"], P, S, H, D, T, r, n_groups, metric, mask, idx, na, vc, ws, ws_bytes, stream=sq)
     vs = new()

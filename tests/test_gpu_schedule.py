@@ -47,9 +47,9 @@ def test_schedule_driver_against_oracle():
         torch.cuda.synchronize()
         _, sent = binding.layer_step(step, total, warmup, interval, dev(prev_v) if prev_v is not None else d["v"],
                                      d["q"], d["k"], d["v"], wq, wk, cfg["eps"], cs, P, S, H, D, T, n_groups,
-                                     metric, mask, idx, na, comp["q"].t, comp["k"].t, comp["v"].t,
+                                     metric, mask, idx, na, *([None] * 3 if step % 2 else [comp[x].t for x in "qkv"]),
                                      cache["q"].t, cache["k"].t, cache["v"].t, ws, ws_bytes,
-                                     order=binding.V_FIRST, stream_qk=sq, stream_v=sv)
+                                     order=binding.V_FIRST, stream_qk=sq, stream_v=sv)     # odd steps: direct delivery
         sq.synchronize()
         exact = dict(zip("qkv", oracle.prologue(cur["q"], cur["k"], cur["v"], seq.wq, seq.wk, cfg["eps"], cs_ref, P)))
         if full:

@@ -139,6 +139,53 @@ def test_selective_prologue_full_size(order, two_streams, T, n_groups, r):
         g.cache[x].assert_guards(x + " cache")
 
 
+@pytest.mark.parametrize("order,two_streams", ORDERS, ids=["lump", "v_first_two_streams", "v_first_one_stream"])
+@pytest.mark.parametrize("T,n_groups", [(64, 1), (1, 24)], ids=["tiles64", "per_token_per_rank"])
+def test_selective_prologue_direct_delivery_full_size(order, two_streams, T, n_groups):
+    """Direct delivery (no compact buffers: the active rows go straight to the caches) at
+    the size the benchmark times, three calls back to back, against the oracle."""
+    d, g = _data(), _Device.get()
+    cfg = d["cfg"]
+    P, S, H, D, r = cfg["P"], cfg["S"], cfg["H"], cfg["D"], 0.8
+    n = S // T
+    want = _expected(T, n_groups, r)
+    ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
+    for x in "qkv":
+        g.comp[x].t.fill_(0x5A5A)
+        g.cache[x].t.copy_(g.old[x])
+    g.metric.fill_(-1)
+    g.mask.fill_(9)
+    g.idx.fill_(-1)
+    g.na.fill_(-1)
+    sq = g.sq
+    sv = g.sv if two_streams else sq
+    torch.cuda.synchronize()
+    for _ in range(3):
+        binding.selective_prologue(g.prev_v, g.q, g.k, g.v, g.wq, g.wk, cfg["eps"], g.cs, P, S, H, D, T, r, n_groups,
+                                   g.metric, g.mask, g.idx, g.na, None, None, None,
+                                   g.cache["q"].t, g.cache["k"].t, g.cache["v"].t, g.ws, ws_bytes,
+                                   order=order, stream_qk=sq, stream_v=sv)
+    sq.synchronize()
+    na = want["na"]
+    assert np.array_equal(g.metric.cpu().numpy().view(np.uint64)[:n], want["metric"])
+    assert int(g.na.item()) == na
+    assert np.array_equal(g.mask.cpu().numpy()[:n], want["mask"])
+    assert np.array_equal(g.idx.cpu().numpy()[:na], want["idx"])
+    tok = (want["idx"][:, None].astype(np.int64) * T + np.arange(T)[None, :]).reshape(-1)
+    inactive = np.ones(S, bool)
+    inactive[tok] = False
+    for x in "qkv":
+        cache_ref = want["cache"][x]
+        got = g.cache[x].host((H, S, D))
+        assert np.array_equal(got[:, inactive], cache_ref[:, inactive]), f"{x}: cached rows must not move"
+        if x == "v":
+            assert np.array_equal(got, cache_ref)
+        else:
+            f = np.ascontiguousarray(d["ref_f"][x][tok].transpose(1, 0, 2))
+            assert_norm_rope_close(got[:, tok], cache_ref[:, tok], f, f"{x} cache, direct delivery")
+        g.cache[x].assert_guards(x + " cache")
+
+
 def test_layer_step_schedule_full_size():
     """The first 12 steps of the paper's 50-step schedule (5 warm-up steps, refresh every
     10, linear cache ratio) on the full temporal workload, step by step against the oracle.
@@ -173,9 +220,9 @@ def test_layer_step_schedule_full_size():
         torch.cuda.synchronize()
         _, sent = binding.layer_step(step, total, warmup, interval, dev(prev_v) if prev_v is not None else d["v"],
                                      d["q"], d["k"], d["v"], wq, wk, cfg["eps"], cs, P, S, H, D, T, n_groups,
-                                     metric, mask, idx, na, comp["q"].t, comp["k"].t, comp["v"].t,
+                                     metric, mask, idx, na, *([None] * 3 if step % 2 else [comp[x].t for x in "qkv"]),
                                      cache["q"].t, cache["k"].t, cache["v"].t, ws, ws_bytes,
-                                     order=order, stream_qk=sq, stream_v=s_v)
+                                     order=order, stream_qk=sq, stream_v=s_v)       # odd steps: direct delivery
         sq.synchronize()
         normed, normed_f = {"v": cur["v"]}, {}
         for x, w in (("q", seq.wq), ("k", seq.wk)):

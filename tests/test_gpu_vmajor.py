@@ -409,3 +409,81 @@ def test_selective_prologue_random_small_shapes():
             assert np.all(comp[t].host()[comp_ref.size:] == 0x5A5A), what
             comp[t].assert_guards()
             cache[t].assert_guards()
+
+
+def _direct_cases():
+    cases = [(4, 768, 4, 64, 16, 0.8, 1), (2, 256, 6, 128, 1, 0.5, 2), (3, 99, 3, 32, 11, 0.0, 1),
+             (2, 384, 2, 256, 64, 1.0, 1), (4, 2400, 4, 40, 1, 0.8, 1), (2, 1024, 8, 128, 256, 0.5, 1)]
+    rng = np.random.default_rng(311)
+    for _ in range(12):
+        P = int(rng.choice([1, 2, 3, 4, 6]))
+        H = P * int(rng.integers(1, 4))
+        D = int(rng.choice([8, 24, 32, 48, 64, 104, 128, 200, 256]))
+        T = int(rng.choice([1, 2, 3, 5, 16, 64]))
+        S = P * T * int(rng.integers(1, 40 if T < 16 else 6))
+        n = S // T
+        cases.append((P, S, H, D, T, float(rng.choice([0.0, 1.0, 0.5, 0.8, rng.random()])),
+                      int(rng.choice([g for g in (1, 2, P, n) if n % g == 0]))))
+    return cases
+
+
+def test_selective_prologue_direct_delivery():
+    """Without compact buffers the active rows go straight to the caches: the caches
+    match the oracle's select -> extract -> scatter and carry the very bits the call with
+    compact buffers leaves there; selection outputs are the same; nothing else is touched."""
+    orders = [(binding.LUMP, False), (binding.V_FIRST, True), (binding.V_FIRST, False)]
+    for case, (P, S, H, D, T, r, n_groups) in enumerate(_direct_cases()):
+        order, two = orders[case % 3]
+        what = dict(case=case, P=P, S=S, H=H, D=D, T=T, r=r, n_groups=n_groups, order=order, two_streams=two)
+        E, n = S * H * D, S // T
+        rng = np.random.default_rng(900 + case)
+        prev, cur_v, _ = _pair(S, H, D, T, seed=500 + case)
+        x = {"q": synth.normal_bf16(40 + case, "q", E).reshape(S, H, D),
+             "k": synth.normal_bf16(40 + case, "k", E).reshape(S, H, D), "v": cur_v}
+        w = {"q": synth.normal_bf16(40 + case, "wq", D, 1.0, 0.1), "k": synth.normal_bf16(40 + case, "wk", D, 1.0, 0.1)}
+        pos = rng.integers(0, 150, (S, 2)).astype(np.int32)
+        cs_ref, cs = oracle.rope_table_2d(pos, D, 10000.0), rope_table(pos, D, 10000.0)
+        old = {t: synth.normal_bf16(9, "old" + t, E).reshape(H, S, D) for t in "qkv"}
+        d = {t: dev(x[t]) for t in "qkv"}
+        sq = torch.cuda.Stream()
+        sv = torch.cuda.Stream() if two else sq
+        runs = {}
+        for mode in ("compact", "direct"):
+            comp = {t: Guarded(E) for t in "qkv"}
+            cache = {t: Guarded(E, fill=old[t]) for t in "qkv"}
+            sel = Selector(P, S, H, D, T)
+            cb = [comp[t].t if mode == "compact" else None for t in "qkv"]
+            torch.cuda.synchronize()
+            for _ in range(2):
+                binding.selective_prologue(dev(prev), d["q"], d["k"], d["v"], dev(w["q"]), dev(w["k"]), 1e-6, cs,
+                                           P, S, H, D, T, r, n_groups, sel.metric, sel.mask, sel.idx, sel.n_active,
+                                           *cb, cache["q"].t, cache["k"].t, cache["v"].t, sel.ws, sel.ws_bytes,
+                                           order=order, stream_qk=sq, stream_v=sv)
+            sq.synchronize()
+            runs[mode] = (sel, comp, cache)
+        m_ref = oracle.vmajor_metric(prev, cur_v, P, T)
+        mask_ref, idx_ref, na_ref = oracle.vmajor_select(m_ref, n_groups, r)
+        sel, comp, cache = runs["direct"]
+        assert np.array_equal(sel.metric.cpu().numpy().view(np.uint64)[:n], m_ref), what
+        assert int(sel.n_active.item()) == na_ref, what
+        assert np.array_equal(sel.mask.cpu().numpy()[:n], mask_ref), what
+        assert np.array_equal(sel.idx.cpu().numpy()[:na_ref], idx_ref), what
+        tok = (idx_ref[:, None] * T + np.arange(T)[None, :]).reshape(-1).astype(np.int64)
+        untouched = np.ones(S, bool)
+        untouched[tok] = False
+        for t in "qkv":
+            if t == "v":
+                ref, ref_f = x["v"], None
+            else:
+                ref, ref_f = oracle.norm_rope(x[t], w[t], 1e-6, cs_ref, want_f32=True)
+            want_cache = oracle.unpack(oracle.pack_active(ref, idx_ref, P, T), idx_ref, old[t].copy(), P, T)
+            got = cache[t].host((H, S, D))
+            assert np.array_equal(got[:, untouched], want_cache[:, untouched]), what
+            if t == "v":
+                assert np.array_equal(got, want_cache), what
+            elif na_ref:
+                assert_norm_rope_close(got[:, tok], want_cache[:, tok],
+                                       np.ascontiguousarray(ref_f[tok].transpose(1, 0, 2)), f"{t} {what}")
+            assert np.array_equal(got, runs["compact"][2][t].host((H, S, D))), "both modes leave the same bits"
+            assert np.all(comp[t].host() == 0x5A5A), "no compact buffer is written"
+            cache[t].assert_guards()
