@@ -30,7 +30,7 @@ using namespace rows;
 // 4 blocks per SM (<= 64 registers), evict-first accesses; heads per block and
 // loads in flight per thread depend on what the launch contains.
 constexpr int kThreads = 256, kMinBlocks = 4;
-// heads per item of the selective mover (items of 2 to 24 heads measured: 6 and 12 are the fastest)
+// selective mover: rows (heads) requested from the L2 ahead, and the least heads worth a block of its own
 constexpr int kSelHeads = 6;
 
 // Grid: one block per (head range, job, token tile); THREADS x MINB = threads resident per SM.
@@ -51,8 +51,13 @@ __global__ void __launch_bounds__(kThreads, kMinBlocks) move_rows_kernel(const _
     if (p.pdl & PDL_WAIT_AT_END) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// The selective mover: 4 blocks of 256 threads per SM.  (One block of 1024 threads ranks the
+// units once per SM instead of four times and is 0.4 us faster on 64-token tiles, but slower on
+// per-token units and at low cache ratios.)
+constexpr int kSelThreads = kThreads, kSelBlocks = kMinBlocks;
+
 template <int LPR, bool PAD>
-__global__ void __launch_bounds__(kThreads, kMinBlocks)
+__global__ void __launch_bounds__(kSelThreads, kSelBlocks)
 selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constant__ SelectParams sel, const int select_here) {
     __shared__ vmajor::SmallSel sm;
     if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -60,7 +65,7 @@ selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constan
     const int32_t *list = p.idx;
     long long nv;
     if (select_here) {
-        nv = (long long)vmajor::select_small<kThreads>(sel, 0, sel.n, sm, blockIdx.x == 0) * p.T;
+        nv = (long long)vmajor::select_small<kSelThreads>(sel, 0, sel.n, sm, blockIdx.x == 0) * p.T;
         list = sm.idx;
     } else if (p.map == MAP_FULL || p.slots_exact) {
         nv = p.n_slots;  // every slot moves: a plain move, or a grid sized from the rule's own count
@@ -69,16 +74,25 @@ selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constan
     }
     int n_valid = nv < (long long)p.n_slots ? (int)nv : p.n_slots;
     if (n_valid < 0) n_valid = 0;
-    // One resident wave of blocks walks the (head range, tensor, token tile) items, so that a
-    // block ranks the units once however many items it moves.  Only the tiles that hold active
-    // slots are walked (the grid's capacity may be larger: the host need not know n_active).
-    constexpr unsigned TOK = kThreads / LPR;
-    const unsigned tiles_cap = ((unsigned)p.n_slots + TOK - 1) / TOK;
+    // One resident wave of blocks, so that a block ranks the units once whatever it moves.  The
+    // work - for every tensor and every token tile that holds active slots, the H heads - is cut
+    // into gridDim.x equal contiguous runs of (tensor, tile, head) rows, heads fastest: a block
+    // meets at most two tiles more than its share of heads spans, and no block has more than one
+    // head row (of TOK tokens) more than another.  Only the tiles that hold active slots count
+    // (the grid's capacity may be larger: the host need not know n_active).
+    constexpr unsigned TOK = kSelThreads / LPR;
     const unsigned tiles = ((unsigned)n_valid + TOK - 1) / TOK;
-    const unsigned groups = (unsigned)p.head_split * (unsigned)p.njobs;   // (head range, tensor) pairs
-    for (unsigned item = blockIdx.x; item < tiles * groups; item += gridDim.x) {
-        const unsigned grp = item / tiles, tile = item - grp * tiles;
-        move_block<LPR, PAD, KIND_MIXED, 4, 4, kThreads, true, kSelHeads>(p, grp * tiles_cap + tile, list, n_valid);
+    const unsigned long long total = (unsigned long long)tiles * (unsigned)p.njobs * (unsigned)p.H;
+    const unsigned long long per = (total + gridDim.x - 1) / gridDim.x;
+    unsigned long long at = per * blockIdx.x;
+    const unsigned long long end = at + per < total ? at + per : total;
+    while (at < end) {
+        const unsigned pair = (unsigned)(at / (unsigned)p.H);        // (tensor, tile), tensor-major
+        const int h_lo = (int)(at - (unsigned long long)pair * (unsigned)p.H);
+        const int h_hi = (unsigned long long)(p.H - h_lo) < end - at ? p.H : h_lo + (int)(end - at);
+        const unsigned job_i = pair / tiles, tile = pair - job_i * tiles;
+        move_range<LPR, PAD, KIND_MIXED, 4, 4, kSelThreads, true, kSelHeads>(p, job_i, tile, h_lo, h_hi, list, n_valid);
+        at += (unsigned)(h_hi - h_lo);
     }
 }
 
@@ -139,12 +153,24 @@ cudaError_t launch_lpr(MoveParams p, cudaStream_t stream) {
 template <int LPR, bool PAD>
 cudaError_t launch_selective_lpr(MoveParams p, const SelectParams *sel, cudaStream_t stream) {
     static const SelectParams none = {};
-    // items of 6 heads: fine enough to balance one resident wave (4 blocks on each SM)
-    const long long items = grid_blocks(p, LPR, kSelHeads);
-    if (items > 0xffffffffLL) return cudaErrorInvalidConfiguration;
-    const long long wave = (long long)sm_count() * kMinBlocks;
-    return launch_grid(selective_move_kernel<LPR, PAD>, items < wave ? items : wave, stream, p.pdl, p, sel ? *sel : none,
-                       sel ? 1 : 0);
+    // one resident wave, but no more blocks than runs of kSelHeads heads
+    constexpr int tok = kSelThreads / LPR;
+    const long long tiles = ((long long)p.n_slots + tok - 1) / tok;
+    const long long rows = tiles * p.njobs * p.H;
+    const long long most = (rows + kSelHeads - 1) / kSelHeads;
+    const long long wave = (long long)sm_count() * kSelBlocks;
+    p.head_split = 1;
+    if (most == 0) return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(most < wave ? most : wave));
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (p.pdl & PDL_LAUNCH_ATTR) ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, selective_move_kernel<LPR, PAD>, p, sel ? *sel : none, sel ? 1 : 0);
 }
 
 // D = 8 * lanes; a lane group is padded to the next power of two.

@@ -61,7 +61,7 @@ __device__ __forceinline__ void heads_loop(int &h, const int h_hi, F &&body) {
     if constexpr (U > 1) heads_loop<U / 2>(h, h_hi, body);
 }
 
-// One block's share of a move: block id b -> (head range, job, token tile).
+// Heads [h_lo, h_hi) of one token tile of one tensor (job).
 // A row of D bf16 values is D/8 16-byte vectors, one per lane of an LPR-lane
 // group (LPR a power of two).  PAD = false: D = 8 * LPR; PAD = true: D/8 < LPR and
 // the lanes beyond the row neither load nor store (they add zero to the row's
@@ -73,33 +73,19 @@ __device__ __forceinline__ void heads_loop(int &h, const int h_hi, F &&body) {
 // memory) and n_valid (active token slots) are resolved by the calling kernel.
 // PF: source rows (heads) requested from the L2 ahead of the block's own loads.
 template <int LPR, bool PAD, int KIND, int UN, int UP, int THREADS, bool DUAL, int PF = 0>
-__device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b, const int32_t *idx_list,
-                                           const int n_valid) {
+__device__ __forceinline__ void move_range(const MoveParams &p, const unsigned job_i, const unsigned tile, const int h_lo,
+                                           const int h_hi, const int32_t *idx_list, const int n_valid) {
     constexpr int TOK = THREADS / LPR;  // token slots per tile
     const int D = PAD ? p.D : LPR * 8;
 
     long long src_head = p.src_head, dst_head = p.dst_head;
     if (src_head == COMPACT_STRIDE) src_head = (long long)n_valid * D;
     if (dst_head == COMPACT_STRIDE) dst_head = (long long)n_valid * D;
-    // Block id -> (head range, job, token tile), head-range-major: the V, Q and K
-    // tiles of one head range are neighbours in the grid, so V's plain blocks run
-    // beside the arithmetic-heavier Q/K blocks.
-    const unsigned tiles = (unsigned)(p.n_slots + TOK - 1) / TOK;
-    const unsigned hsplit = (unsigned)p.head_split, njobs = (unsigned)p.njobs;
-    const unsigned y = b / (tiles * njobs);
-    const unsigned rem = b - y * tiles * njobs;
-    const unsigned job_i = rem / tiles;
-    const unsigned tile = rem - job_i * tiles;
     const int tile0 = (int)tile * TOK;
     if (tile0 >= n_valid) return;  // block-uniform: nothing in this tile
     const long long sh = src_head / 8, dh = dst_head / 8;  // head strides in vectors
     const int lr = (int)threadIdx.x % LPR;
     const bool lane_on = !PAD || lr < D / 8;
-
-    // heads [h_lo, h_hi) of this block
-    const int hs = (p.H + (int)hsplit - 1) / (int)hsplit;
-    const int h_lo = (int)y * hs;
-    const int h_hi = h_lo + hs < p.H ? h_lo + hs : p.H;
     const MoveJob job = job_i == 0 ? p.job[0] : (job_i == 1 ? p.job[1] : p.job[2]);
 
     // A slot past the end keeps its lanes in step with the warp (the row
@@ -241,6 +227,26 @@ __device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b
             }
         }
     });
+}
+
+// One block's share of a grid of one block per (head range, job, token tile):
+// block id b, head-range-major, so that the V, Q and K tiles of one head range are
+// neighbours in the grid and V's plain blocks run beside the arithmetic-heavier
+// Q/K blocks.
+template <int LPR, bool PAD, int KIND, int UN, int UP, int THREADS, bool DUAL>
+__device__ __forceinline__ void move_block(const MoveParams &p, const unsigned b, const int32_t *idx_list,
+                                           const int n_valid) {
+    constexpr int TOK = THREADS / LPR;
+    const unsigned tiles = (unsigned)(p.n_slots + TOK - 1) / TOK;
+    const unsigned hsplit = (unsigned)p.head_split, njobs = (unsigned)p.njobs;
+    const unsigned y = b / (tiles * njobs);
+    const unsigned rem = b - y * tiles * njobs;
+    const unsigned job_i = rem / tiles;
+    const unsigned tile = rem - job_i * tiles;
+    const int hs = (p.H + (int)hsplit - 1) / (int)hsplit;
+    const int h_lo = (int)y * hs;
+    const int h_hi = h_lo + hs < p.H ? h_lo + hs : p.H;
+    move_range<LPR, PAD, KIND, UN, UP, THREADS, DUAL>(p, job_i, tile, h_lo, h_hi, idx_list, n_valid);
 }
 
 }  // namespace rows

@@ -73,7 +73,7 @@ __device__ __forceinline__ unsigned long long unit_metric(const SelectParams &p,
 // are active.  Leaves the ascending active list in sm.idx and returns its
 // length; with publish the block also writes metric_out, mask, idx and n_active.
 constexpr int kStageMax = 768;   // piece sums staged at once (units * pieces of the selections that run in a consumer)
-struct SmallSel {
+struct alignas(16) SmallSel {
     unsigned long long m[kCountMax];
     unsigned long long stage[kStageMax];
     int idx[kCountMax];
@@ -113,28 +113,36 @@ __device__ int select_small(const SelectParams &p, const int base, const int cnt
     for (int e = tid; e < cnt; e += BLOCK)
         if (sm.m[e] >> 55) sm.wide = 1;
     __syncthreads();
+    static_assert(BLOCK >= kCountMax, "one thread per unit");
+    const int e = tid;
     if (!sm.wide) {
-        for (int e = tid; e < cnt; e += BLOCK) sm.stage[e] = (sm.m[e] << 9) | (unsigned long long)e;  // cnt <= 256 < 2^9
+        if (e < cnt) sm.stage[e] = (sm.m[e] << 9) | (unsigned long long)e;  // cnt <= 256 < 2^9
         __syncthreads();
-        for (int e = tid; e < cnt; e += BLOCK) {
-            const int g0 = (e / p.g) * p.g;  // base is a multiple of g
+        if (e < cnt) {
+            const int g0 = (e / p.g) * p.g, g1 = g0 + p.g;  // base is a multiple of g
             const unsigned long long my = sm.stage[e];
             int rank = 0;
+            // every warp reads every key of its units' groups, so the loop is bound by the
+            // shared-memory pipe: two keys per load
+            int j = g0;
+            if ((j & 1) && j < g1) rank += sm.stage[j++] < my;
 #pragma unroll 4
-            for (int j = g0; j < g0 + p.g; ++j) rank += sm.stage[j] < my;
-            sm.active[e] = rank >= p.n_cached ? 1 : 0;
-        }
-    } else {
-        for (int e = tid; e < cnt; e += BLOCK) {
-            const int g0 = (e / p.g) * p.g;
-            const unsigned long long my = sm.m[e];
-            int rank = 0;
-            for (int j = g0; j < g0 + p.g; ++j) {
-                const unsigned long long o = sm.m[j];
-                rank += (o < my) | ((o == my) & (j < e));
+            for (; j + 2 <= g1; j += 2) {
+                const ulonglong2 kk = *reinterpret_cast<const ulonglong2 *>(&sm.stage[j]);
+                rank += (kk.x < my) + (kk.y < my);
             }
+            if (j < g1) rank += sm.stage[j] < my;
             sm.active[e] = rank >= p.n_cached ? 1 : 0;
         }
+    } else if (e < cnt) {
+        const int g0 = (e / p.g) * p.g;
+        const unsigned long long my = sm.m[e];
+        int rank = 0;
+        for (int j = g0; j < g0 + p.g; ++j) {
+            const unsigned long long o = sm.m[j];
+            rank += (o < my) | ((o == my) & (j < e));
+        }
+        sm.active[e] = rank >= p.n_cached ? 1 : 0;
     }
     __syncthreads();
     const int cnt_pad = (cnt + 31) / 32 * 32;
