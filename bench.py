@@ -358,9 +358,13 @@ def run_ours(args):
     step_bytes = algorithmic_bytes(cfg)
     peak, peak_kind = measured_peak()
 
-    def step(order):
+    # The headline is V-first on ONE stream: V's launch, then Q/K's as its programmatic dependent; and a
+    # call's first kernel is the programmatic dependent of the previous call's last one, so consecutive
+    # layers overlap launch, ramp-up and drain while every kernel still waits for its predecessor
+    # before it touches memory.  (The same order on two streams, joined by events, is a row of `orders`.)
+    def step(order, two_streams=False):
         binding.prologue(q, k, v, qh, kh, vh, wq, wk, cfg["eps"], cs, P, S, H, D, order=order,
-                         stream_qk=sq, stream_v=sv)
+                         stream_qk=sq, stream_v=sv if two_streams else sq)
 
     def barrier():
         torch.cuda.synchronize()
@@ -417,20 +421,18 @@ def run_ours(args):
     elif rank == 0:
         # ---- per-order detail, per-step events (this GPU only) --------------
         orders = {}
-        for name, order in (("v_first", binding.V_FIRST), ("lump", binding.LUMP)):
-            ms = time_steps(torch, lambda: step(order), sq, args.steps, 3)
+        for name, order, two in (("v_first", binding.V_FIRST, False), ("v_first_two_streams", binding.V_FIRST, True),
+                                 ("lump", binding.LUMP, False)):
+            ms = time_steps(torch, lambda: step(order, two), sq, args.steps, 3)
+            loop = [time_loop(torch, lambda: step(order, two), sq, rep_steps) for _ in range(5)]
             orders[name] = {"us_median": 1e3 * statistics.median(ms), "us_min": 1e3 * min(ms),
                             "gbs_median": step_bytes / (statistics.median(ms) * 1e-3) / 1e9,
+                            "us_back_to_back_median": 1e3 * statistics.median(loop), "us_back_to_back_min": 1e3 * min(loop),
+                            "gbs_back_to_back": step_bytes / (statistics.median(loop) * 1e-3) / 1e9,
                             "launches_per_step": 2 if order == binding.V_FIRST else 1}
-
-        def one_stream():
-            binding.prologue(q, k, v, qh, kh, vh, wq, wk, cfg["eps"], cs, P, S, H, D, order=binding.V_FIRST,
-                             stream_qk=sq, stream_v=sq)
-        ms1 = [time_loop(torch, one_stream, sq, rep_steps) for _ in range(5)]
-        orders["v_first_one_stream"] = {"us_back_to_back_median": 1e3 * statistics.median(ms1), "us_back_to_back_min": 1e3 * min(ms1),
-                                        "gbs_median": step_bytes / (statistics.median(ms1) * 1e-3) / 1e9, "launches_per_step": 2,
-                                        "note": "V's launch, then Q/K's with a programmatic dependent launch (no events); "
-                                                "timed like `repeats`"}
+        orders["note"] = ("us_median: one call between two events; us_back_to_back: the loop of `repeats`.  v_first = V's launch, "
+                          "then Q/K's as its programmatic dependent on one stream (the headline); v_first_two_streams = the same "
+                          "two launches on two streams joined by events (no dependent launches across the join)")
         # V-first evidence: V's exchange and the Q/K launch issued as two calls with their own events
         ev = {n: torch.cuda.Event(enable_timing=True) for n in ("v0", "v1", "qk0", "qk1")}
         timeline = []
@@ -526,6 +528,7 @@ def run_ours(args):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "storage_dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "P": P, "S": S, "H": H, "D": D, "order": "v_first",
+                       "streams": "one: V's launch, then Q/K's as its programmatic dependent; consecutive calls are chained the same way",
                        "algorithmic_bytes_per_step": step_bytes, "l2": "inputs and outputs (775 MB per step) exceed the 126 MB L2",
                        "replicas": world},
             "gpu_launches": 2 * args.steps,
@@ -594,6 +597,10 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
     floor = launch_floor(torch, binding, sq, flush, iters)
     out["launch_floor"] = {"us": floor, "what": "median event-to-event time of one prologue launch that moves 8 KB, same "
                                                 "flush-and-events protocol: the fixed cost inside every per_config figure"}
+    # v_first: V's launch, then Q/K's as its programmatic dependent, on one stream (consecutive calls chain
+    # the same way: best back to back); v_first_two_streams: the two launches start side by side on two
+    # streams joined by events (best for a single call between two events); lump: one launch
+    ORDERS3 = (("v_first", binding.V_FIRST, False), ("v_first_two_streams", binding.V_FIRST, True), ("lump", binding.LUMP, False))
     for name in names:
         cfg = synth.config(name)
         P, S, H, D = cfg["P"], cfg["S"], cfg["H"], cfg["D"]
@@ -605,18 +612,18 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
         binding.rope_table_2d(cs, dev(L["pos"], torch), S, D, cfg["theta"])
         qh, kh, vh = (torch.empty(E, dtype=torch.int16, device="cuda") for _ in range(3))
 
-        def full(order):
+        def full(order, two=False):
             binding.prologue(q, k, v, qh, kh, vh, wq, wk, cfg["eps"], cs, P, S, H, D,
-                             order=order, stream_qk=sq, stream_v=sv)
+                             order=order, stream_qk=sq, stream_v=sv if two else sq)
         b = algorithmic_bytes(cfg)
         out[name] = {"bytes": b, "fits_in_l2": b < 126e6 * 2}
-        for oname, order in (("v_first", binding.V_FIRST), ("lump", binding.LUMP)):
-            cold_all = time_steps(torch, lambda: full(order), sq, iters, 10, flush=flush)
+        for oname, order, two in ORDERS3:
+            cold_all = time_steps(torch, lambda: full(order, two), sq, iters, 10, flush=flush)
             cold = statistics.median(cold_all)
-            warm = statistics.median(time_steps(torch, lambda: full(order), sq, iters, 10))
+            warm = statistics.median(time_steps(torch, lambda: full(order, two), sq, iters, 10))
             out[name][oname] = {"us_cold_l2": 1e3 * cold, "us_cold_l2_min": 1e3 * min(cold_all), "iterations": iters,
                                 "gbs_effective_cold_l2": b / (cold * 1e-3) / 1e9, "us_warm_l2": 1e3 * warm}
-            gr = time_graph(torch, lambda: full(order), sq, iters, flush=flush)
+            gr = time_graph(torch, lambda: full(order, two), sq, iters, flush=flush)
             if gr is not None:
                 out[name][oname]["us_cold_l2_cuda_graph"] = 1e3 * statistics.median(gr)
         if name != "temporal":
@@ -625,14 +632,14 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
             # reads from HBM and the write-back of its output falls inside the timed region.
             n_sets = max(2, min(64, int(np.ceil(4 * 126e6 / b)) + 1))
             sets = [([t.clone() for t in (q, k, v)], [torch.empty_like(qh) for _ in range(3)]) for _ in range(n_sets)]
-            for oname, order in (("v_first", binding.V_FIRST), ("lump", binding.LUMP)):
+            for oname, order, two in ORDERS3:
                 calls = [0]
 
                 def rotating():
                     (a, c, d), (x, y, z) = sets[calls[0] % n_sets]
                     calls[0] += 1
                     binding.prologue(a, c, d, x, y, z, wq, wk, cfg["eps"], cs, P, S, H, D, order=order,
-                                     stream_qk=sq, stream_v=sv)
+                                     stream_qk=sq, stream_v=sv if two else sq)
                 ms = time_graph_loop(torch, rotating, sq, n_sets, replays=10)
                 if ms is None:
                     continue

@@ -17,6 +17,15 @@
  *     synchronises the device and enqueues only on the streams it is given
  *     (void* = cudaStream_t, NULL = the default stream).  Calls return as soon
  *     as the work is enqueued.
+ *   - Stream order holds between calls and towards the caller's own work.  On
+ *     one stream the first kernel of a call is launched with programmatic
+ *     stream serialization and waits (griddepcontrol.wait) for whatever
+ *     precedes it before it touches memory, and the last kernel of a call lets
+ *     its successor become resident while it drains, so consecutive calls
+ *     overlap launch latency, ramp-up and drain.  A kernel of the caller that
+ *     follows a call is not affected unless the caller launches it with the
+ *     same attribute; it then has to call cudaGridDependencySynchronize()
+ *     before it reads the call's outputs, as the programming model requires.
  *   - bf16 tensors are passed as uint16_t bit patterns, row-major, last index
  *     fastest, and must be 16-byte aligned.  Head dimension D is a multiple of
  *     8 from 8 to 256 (a row is D/8 16-byte vectors, one per lane of a group of

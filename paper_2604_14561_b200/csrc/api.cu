@@ -123,6 +123,13 @@ MoveParams seq_to_head(int S, int H, int D) {
 }
 
 // Shared by cocodiff_ulysses_a2a (no weights) and cocodiff_prologue.
+// A call's first kernel is launched with the programmatic attribute and waits for its
+// predecessor in the stream before it touches memory; its last kernel lets whatever follows
+// become resident while it drains.  Consecutive calls on one stream (layer after layer) then
+// overlap launch latency, ramp-up and drain without giving up their order; a successor that
+// was launched without the attribute starts when the last kernel has completed, as ever.
+constexpr int kChainedLaunch = PDL_LAUNCH_ATTR | PDL_WAIT_AT_START | PDL_TRIGGER;
+
 int exchange(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *qh, uint16_t *kh,
              uint16_t *vh, const uint16_t *wq, const uint16_t *wk, float eps, const float *cs, int S,
              int H, int D, int order, cudaStream_t sq, cudaStream_t sv) {
@@ -136,11 +143,11 @@ int exchange(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *
         // waits for V's grid only before it completes (the stream's order of completion holds).
         MoveParams pv = base;
         pv.job[pv.njobs++] = MoveJob{v, vh, nullptr, nullptr};
-        pv.pdl = PDL_TRIGGER;
+        pv.pdl = kChainedLaunch;  // Q/K's launch follows once V's blocks have passed their wait
         MoveParams pqk = base;
         if (q) pqk.job[pqk.njobs++] = MoveJob{q, qh, wq, nullptr};
         if (k) pqk.job[pqk.njobs++] = MoveJob{k, kh, wk, nullptr};
-        pqk.pdl = PDL_LAUNCH_ATTR | PDL_WAIT_AT_END;
+        pqk.pdl = PDL_LAUNCH_ATTR | PDL_WAIT_AT_END | PDL_TRIGGER;
         CK(launch_move(pv, sq));
         CK(launch_move(pqk, sq));
         return COCODIFF_OK;
@@ -152,6 +159,7 @@ int exchange(const uint16_t *q, const uint16_t *k, const uint16_t *v, uint16_t *
         if (q) p.job[p.njobs++] = MoveJob{q, qh, wq, nullptr};
         if (k) p.job[p.njobs++] = MoveJob{k, kh, wk, nullptr};
         if (p.njobs == 0) return COCODIFF_OK;
+        p.pdl = kChainedLaunch;
         CK(launch_move(p, sq));
         return COCODIFF_OK;
     }
@@ -329,6 +337,7 @@ int enqueue_pack(const uint16_t *const in[3], uint16_t *const out[3], const uint
                  int H, int D, int T, cudaStream_t st) {
     MoveParams p = make_pack_params(in, out, nullptr, wq, wk, eps, cs, idx, n_active, slots, S, H, D, T);
     if (p.njobs == 0) return COCODIFF_OK;
+    p.pdl = kChainedLaunch;
     CK(launch_selective_move(p, nullptr, st));  // a resident wave that walks the active tiles only
     return COCODIFF_OK;
 }
@@ -345,12 +354,12 @@ int enqueue_select_and_pack(const SelectionPlan &pl, const uint16_t *const in[3]
     // the consuming kernel selects for itself when it has few units to rank and at least one block
     const bool consume = p.njobs > 0 && pl.in_consumer && slots > 0;
     MetricParams mp = pl.mp;
-    mp.pdl = PDL_TRIGGER;
+    mp.pdl = kChainedLaunch;  // the trigger follows the block's loads
     CK(launch_metric(mp, st));
     if (!consume)  // a selection launch: many units, or nothing follows that could select for itself
         CK(launch_select(pl.sp, st, pl.mp.n_units > 0 ? (PDL_LAUNCH_ATTR | PDL_WAIT_AT_START | PDL_TRIGGER) : 0));
     if (p.njobs == 0) return COCODIFF_OK;
-    p.pdl = pl.mp.n_units > 0 ? (PDL_LAUNCH_ATTR | PDL_WAIT_AT_START) : 0;
+    p.pdl = pl.mp.n_units > 0 ? kChainedLaunch : 0;
     CK(launch_selective_move(p, consume ? &pl.sp : nullptr, st));
     return COCODIFF_OK;
 }
@@ -381,6 +390,7 @@ int enqueue_unpack(const uint16_t *const in[3], uint16_t *const out[3], const in
                    const int32_t *n_active, int slots, int S, int H, int D, int T, cudaStream_t st) {
     MoveParams p = make_unpack_params(in, out, idx, n_active, slots, S, H, D, T);
     if (p.njobs == 0) return COCODIFF_OK;
+    p.pdl = kChainedLaunch;
     CK(launch_selective_move(p, nullptr, st));  // a resident wave that walks the active tiles only
     return COCODIFF_OK;
 }
@@ -443,6 +453,7 @@ int cocodiff_qk_norm_rope(const uint16_t *q, const uint16_t *k, uint16_t *q_out,
     if (q) p.job[p.njobs++] = MoveJob{q, q_out, wq};
     if (k) p.job[p.njobs++] = MoveJob{k, k_out, wk};
     if (p.njobs == 0) return COCODIFF_OK;
+    p.pdl = kChainedLaunch;
     CK(launch_move(p, (cudaStream_t)stream));
     return COCODIFF_OK;
 }
@@ -485,6 +496,7 @@ int cocodiff_ulysses_a2a_inverse(const uint16_t *q_head, const uint16_t *k_head,
     for (int i = 2; i >= 0; --i)
         if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr};
     if (p.njobs == 0) return COCODIFF_OK;
+    p.pdl = kChainedLaunch;
     CK(launch_move(p, (cudaStream_t)stream));
     return COCODIFF_OK;
 }
@@ -748,6 +760,7 @@ int cocodiff_selective_prologue(const uint16_t *prev_v, const uint16_t *q, const
     MoveParams p = make_pack_params(in_qk, out_qk, do_unpack ? cache_qk : nullptr, wq, wk, eps, cs, idx, n_active, slots, S,
                                     H, D, T, direct);
     p.slots_exact = 1;
+    p.pdl = kChainedLaunch;
     CK(launch_selective_move(p, nullptr, sq));
     return COCODIFF_OK;
 }
@@ -828,6 +841,7 @@ int cocodiff_tapa_phase1(const uint16_t *q, const uint16_t *k, const uint16_t *v
     for (int i = 2; i >= 0; --i)
         if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr, out[i] + E};
     if (p.njobs == 0) return COCODIFF_OK;
+    p.pdl = kChainedLaunch;
     CK(launch_selective_move(p, nullptr, (cudaStream_t)stream));
     return COCODIFF_OK;
 }

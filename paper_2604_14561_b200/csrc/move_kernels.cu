@@ -36,8 +36,9 @@ constexpr int kSelHeads = 6;
 // Grid: one block per (head range, job, token tile); THREADS x MINB = threads resident per SM.
 template <int LPR, bool PAD, int KIND, int UN, int UP>
 __global__ void __launch_bounds__(kThreads, kMinBlocks) move_rows_kernel(const __grid_constant__ MoveParams p) {
-    if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // wait first: whatever this grid lets start early must not overtake the grid it waits for
     if (p.pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int n_valid = p.n_slots;
     if (p.map != MAP_FULL) {
         // written by an earlier kernel: a coherent load, ordered after griddepcontrol.wait
@@ -60,8 +61,8 @@ template <int LPR, bool PAD>
 __global__ void __launch_bounds__(kSelThreads, kSelBlocks)
 selective_move_kernel(const __grid_constant__ MoveParams p, const __grid_constant__ SelectParams sel, const int select_here) {
     __shared__ vmajor::SmallSel sm;
-    if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (p.pdl & PDL_TRIGGER) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int32_t *list = p.idx;
     long long nv;
     if (select_here) {

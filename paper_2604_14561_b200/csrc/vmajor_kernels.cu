@@ -45,6 +45,7 @@ vmajor_select_large_kernel(const __grid_constant__ SelectParams p, const int mb,
 __global__ void __launch_bounds__(kMetricThreads, kMetricBlocksPerSm)
 vmajor_metric_kernel(const __grid_constant__ MetricParams p) {
     __shared__ unsigned long long warp_part[kMetricThreads / 32];
+    if (p.pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     unsigned long long acc;
     if (p.warp_mode) {
@@ -158,8 +159,7 @@ cudaError_t launch_metric(const MetricParams &p, cudaStream_t stream) {
     if (p.warp_mode) blocks = ((long long)p.n_units + kMetricThreads / 32 - 1) / (kMetricThreads / 32);
     else blocks = (long long)p.n_units * p.parts;
     if (blocks > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    vmajor_metric_kernel<<<(unsigned)blocks, kMetricThreads, 0, stream>>>(p);
-    return cudaGetLastError();
+    return launch_maybe_programmatic(vmajor_metric_kernel, dim3((unsigned)blocks), dim3(kMetricThreads), 0, stream, p.pdl, p);
 }
 
 }  // namespace cocodiff

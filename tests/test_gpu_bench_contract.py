@@ -56,7 +56,7 @@ def test_bench_line_has_every_contract_key():
     assert [row["step"] for row in sel["per_step"]] == list(range(1, 8))
     assert all(row["n_active"] == 29 for row in sel["per_step"]) and sel["n_units"] == 144
     assert sel["algorithmic_bytes"] == 250085376
-    assert 0 < pc["launch_floor"]["us"] < pc["tiny"]["lump"]["us_cold_l2"] + 2.0
+    assert 0 < pc["launch_floor"]["us"] < pc["tiny"]["lump"]["us_cold_l2"] + 4.0
     assert pc["sd3"]["lump"]["back_to_back_rotating_buffers"]["exceeds_4x_l2"] is True
     assert sel["back_to_back_rotating_buffers"]["us_per_step"] > 20.0
     assert set(c["other_workloads_ms_per_layer"]) == {"tiny", "sd3", "qwen768", "temporal"}

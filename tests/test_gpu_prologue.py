@@ -282,3 +282,56 @@ def test_two_host_threads_call_the_library_at_once():
     for t in threads:
         t.join()
     assert not errors, errors
+
+
+@pytest.mark.parametrize("P,S,H,D", [(4, 1000, 8, 128), (24, 9216, 24, 128)])
+def test_calls_chained_on_one_stream_keep_their_order(P, S, H, D):
+    """Consecutive calls on one stream are launched as programmatic dependents of one another
+    (a call's first kernel may become resident while the previous call's last kernel drains).
+    Here every call reads what the call before it wrote, twelve calls without a host
+    synchronisation in between, in both orders of issue: exchange -> inverse -> exchange -> ...
+    must return the input bit for bit, and a stale read anywhere would not."""
+    L, _ = _layer(P, S, H, D, seed=11)
+    E = S * H * D
+    x0 = [dev(L[n]) for n in "qkv"]
+    seq = [[torch.zeros(E, dtype=torch.int16, device="cuda") for _ in range(3)] for _ in range(2)]
+    head = [[torch.zeros(E, dtype=torch.int16, device="cuda") for _ in range(3)] for _ in range(2)]
+    st = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    src = x0
+    for i in range(6):
+        order = binding.V_FIRST if i % 2 == 0 else binding.LUMP
+        binding.ulysses_a2a(*src, *head[i % 2], P, S, H, D, order=order, stream_qk=st, stream_v=st)
+        binding.ulysses_a2a_inverse(*head[i % 2], *seq[i % 2], P, S, H, D, stream=st)
+        src = seq[i % 2]
+    st.synchronize()
+    for n, got in zip("qkv", src):
+        assert np.array_equal(u16(got).reshape(S, H, D), L[n]), n
+    # the selective chain: scatter into the caches, read them back through the inverse, use that as prev_v
+    T, r = (64, 0.5) if S % (P * 64) == 0 else (1, 0.5)      # 144 units ranked inside the mover / 1000 by the selection kernel
+    n_units = S // T
+    wq, wk = dev(L["wq"]), dev(L["wk"])
+    cs = rope_table(L["pos"], D, 10000.0)
+    cache = [torch.zeros(E, dtype=torch.int16, device="cuda") for _ in range(3)]
+    prev_b = torch.zeros(E, dtype=torch.int16, device="cuda")
+    metric = torch.zeros(n_units, dtype=torch.int64, device="cuda")
+    mask = torch.zeros(n_units, dtype=torch.uint8, device="cuda")
+    idx = torch.zeros(n_units, dtype=torch.int32, device="cuda")
+    na = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws_bytes = binding.vmajor_workspace_bytes(P, S, H, D, T)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    binding.prologue(*x0, *cache, wq, wk, 1e-6, cs, P, S, H, D, order=binding.V_FIRST, stream_qk=st, stream_v=st)
+    for i in range(3):
+        binding.ulysses_a2a_inverse(None, None, cache[2], None, None, prev_b, P, S, H, D, stream=st)
+        binding.selective_prologue(prev_b, *x0, wq, wk, 1e-6, cs, P, S, H, D, T, r, 1, metric, mask, idx, na,
+                                   None, None, None, *cache, ws, ws_bytes, order=binding.LUMP, stream_qk=st, stream_v=st)
+    st.synchronize()
+    # prev_b always equalled V exactly (the full step filled the cache, selective steps rewrite the same
+    # bits), so every distance is zero and the rule caches the lowest-numbered half
+    assert np.array_equal(u16(prev_b).reshape(S, H, D), L["v"])
+    assert not metric.any().item()
+    n_cached = int(np.floor(r * n_units))
+    assert int(na.item()) == n_units - n_cached
+    assert np.array_equal(idx.cpu().numpy()[:n_units - n_cached], np.arange(n_cached, n_units))
+    assert np.array_equal(u16(cache[2]).reshape(H, S, D), oracle.ulysses_a2a(L["v"], P))
