@@ -842,7 +842,7 @@ int cocodiff_tapa_phase1(const uint16_t *q, const uint16_t *k, const uint16_t *v
         if (in[i]) p.job[p.njobs++] = MoveJob{in[i], out[i], nullptr, out[i] + E};
     if (p.njobs == 0) return COCODIFF_OK;
     p.pdl = kChainedLaunch;
-    CK(launch_selective_move(p, nullptr, (cudaStream_t)stream));
+    CK(launch_move(p, (cudaStream_t)stream));  // a plain move of whole tensors with two destinations
     return COCODIFF_OK;
 }
 

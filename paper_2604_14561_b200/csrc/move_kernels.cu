@@ -34,7 +34,7 @@ constexpr int kThreads = 256, kMinBlocks = 4;
 constexpr int kSelHeads = 6;
 
 // Grid: one block per (head range, job, token tile); THREADS x MINB = threads resident per SM.
-template <int LPR, bool PAD, int KIND, int UN, int UP>
+template <int LPR, bool PAD, int KIND, int UN, int UP, bool DUAL = false>
 __global__ void __launch_bounds__(kThreads, kMinBlocks) move_rows_kernel(const __grid_constant__ MoveParams p) {
     // wait first: whatever this grid lets start early must not overtake the grid it waits for
     if (p.pdl & PDL_WAIT_AT_START) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(kThreads, kMinBlocks) move_rows_kernel(const _
         n_valid = nv < (long long)p.n_slots ? (int)nv : p.n_slots;
         if (n_valid < 0) n_valid = 0;
     }
-    move_block<LPR, PAD, KIND, UN, UP, kThreads, false>(p, blockIdx.x, p.idx, n_valid);
+    move_block<LPR, PAD, KIND, UN, UP, kThreads, DUAL>(p, blockIdx.x, p.idx, n_valid);
     // A grid that started beside its predecessor without consuming its results still has to
     // complete after it: whoever waits for this grid then also has the predecessor's output.
     if (p.pdl & PDL_WAIT_AT_END) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -137,20 +137,6 @@ long long grid_blocks(MoveParams &p, int lpr, int heads_per_block) {
     return tiles * head_split * p.njobs;
 }
 
-// Several blocks per token tile shorten the tail of the grid and let V's plain
-// blocks run beside Q/K's arithmetic-heavier ones (head-range-major block order).
-template <int LPR, bool PAD>
-cudaError_t launch_lpr(MoveParams p, cudaStream_t stream) {
-    int n_norm = 0;
-    for (int i = 0; i < p.njobs; ++i) n_norm += p.job[i].w != nullptr;
-    if (n_norm == 0)  // 4 heads per block, 4-8 rows in flight per thread
-        return launch_grid(move_rows_kernel<LPR, PAD, KIND_PLAIN, 4, 8>, grid_blocks(p, LPR, 4), stream, p.pdl, p);
-    if (n_norm == p.njobs)  // 8 heads per block, 4 rows in flight
-        return launch_grid(move_rows_kernel<LPR, PAD, KIND_NORM, 4, 8>, grid_blocks(p, LPR, 8), stream, p.pdl, p);
-    // V with Q and/or K in one launch: 12 heads per block, 4 rows in flight on both paths
-    return launch_grid(move_rows_kernel<LPR, PAD, KIND_MIXED, 4, 4>, grid_blocks(p, LPR, 12), stream, p.pdl, p);
-}
-
 template <int LPR, bool PAD>
 cudaError_t launch_selective_lpr(MoveParams p, const SelectParams *sel, cudaStream_t stream) {
     static const SelectParams none = {};
@@ -172,6 +158,26 @@ cudaError_t launch_selective_lpr(MoveParams p, const SelectParams *sel, cudaStre
     cfg.attrs = attr;
     cfg.numAttrs = (p.pdl & PDL_LAUNCH_ATTR) ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, selective_move_kernel<LPR, PAD>, p, sel ? *sel : none, sel ? 1 : 0);
+}
+
+// Several blocks per token tile shorten the tail of the grid and let V's plain
+// blocks run beside Q/K's arithmetic-heavier ones (head-range-major block order).
+template <int LPR, bool PAD>
+cudaError_t launch_lpr(MoveParams p, cudaStream_t stream) {
+    int n_norm = 0, n_dual = 0;
+    for (int i = 0; i < p.njobs; ++i) {
+        n_norm += p.job[i].w != nullptr;
+        n_dual += p.job[i].dst2 != nullptr;
+    }
+    if (n_dual != 0)  // whole tensors with two destinations: 8 heads per block (92 -> 84 us against the resident wave)
+        return n_norm == 0 ? launch_grid(move_rows_kernel<LPR, PAD, KIND_PLAIN, 4, 8, true>, grid_blocks(p, LPR, 8), stream, p.pdl, p)
+                           : launch_selective_lpr<LPR, PAD>(p, nullptr, stream);
+    if (n_norm == 0)  // 4 heads per block, 4-8 rows in flight per thread
+        return launch_grid(move_rows_kernel<LPR, PAD, KIND_PLAIN, 4, 8>, grid_blocks(p, LPR, 4), stream, p.pdl, p);
+    if (n_norm == p.njobs)  // 8 heads per block, 4 rows in flight
+        return launch_grid(move_rows_kernel<LPR, PAD, KIND_NORM, 4, 8>, grid_blocks(p, LPR, 8), stream, p.pdl, p);
+    // V with Q and/or K in one launch: 12 heads per block, 4 rows in flight on both paths
+    return launch_grid(move_rows_kernel<LPR, PAD, KIND_MIXED, 4, 4>, grid_blocks(p, LPR, 12), stream, p.pdl, p);
 }
 
 // D = 8 * lanes; a lane group is padded to the next power of two.
