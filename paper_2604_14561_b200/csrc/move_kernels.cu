@@ -15,7 +15,13 @@
 // ranks the units itself from the metric kernel's sums (no selection launch and
 // no one-block stage between the metric pass and the data movement); an active
 // row is then read once and written twice, to the compact send buffer and to its
-// slot of the cached head-parallel tensor.
+// slot of the cached head-parallel tensor (or, without a send buffer, to that
+// slot alone: direct delivery).
+//
+// Programmatic dependent launches: a kernel launched with the attribute waits
+// (griddepcontrol.wait) before it touches memory and only then lets its own
+// successor start, so that nothing it lets start early can overtake the grid it
+// waits for; see PdlFlags.
 #include <mutex>
 
 #include "move_rows.cuh"

@@ -129,10 +129,10 @@ __device__ __forceinline__ void move_range(const MoveParams &p, const unsigned j
     const long long dh2 = DUAL ? p.dst2_head / 8 : 0;
     uint4 *dp2 = DUAL ? reinterpret_cast<uint4 *>(job.dst2 + (dual ? d2 * p.dst2_tok : 0)) + lr + h_lo * dh2 : nullptr;
 
-    // A block that walks a few items of scattered units meets the memory latency anew at every
-    // item (the list, then the per-token constants, then the rows): the rows of the first PF
+    // A block that walks a few runs of scattered units meets the memory latency anew at every
+    // run (the list, then the per-token constants, then the rows): the rows of the first PF
     // heads are asked of the L2 before the constants are loaded.  (Whole-tensor moves and grids
-    // of one item per block hide that latency behind their other work, and measured slower
+    // of one range per block hide that latency behind their other work, and measured slower
     // with the extra requests.)
     if (PF > 0 && p.map != MAP_FULL && lane_on) {
         const int np = h_hi - h_lo < PF ? h_hi - h_lo : PF;
