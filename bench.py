@@ -499,6 +499,15 @@ def run_ours(args):
         per_config = other_configs(torch, binding, args)
         per_config["temporal_steps"] = temporal_rows(torch, binding, args)
         per_config["next_rows_temporal"] = next_rows(torch, binding, args)
+        # the selective step's parts as stand-alone calls (each between two events after an L2 flush, so each
+        # carries the event-to-event floor): what the fused pass replaces
+        nr, ts = per_config["next_rows_temporal"], per_config["temporal_steps"]
+        parts = {"metric_and_selection": ts["metric_pass_context"]["us_metric_and_selection_alone"],
+                 "pack_active_qkv": nr["pack_active_qkv_standalone"]["us_cold_l2"],
+                 "unpack_qkv": nr["unpack_qkv_receiver_only"]["us_cold_l2"]}
+        parts["sum"] = sum(parts.values())
+        parts["fused_step"] = min(ts["steps_1_to_7_selective"]["us_mean"].values())
+        ts["steps_1_to_7_selective"]["break_out_as_stand_alone_calls_us"] = parts
 
         # ---- the oracle on this machine's host cores, bounded sample ------------
         import oracle
