@@ -649,12 +649,13 @@ def other_configs(torch, binding, args, names=("tiny", "sd3", "qwen768", "tempor
                     calls[0] += 1
                     binding.prologue(a, c, d, x, y, z, wq, wk, cfg["eps"], cs, P, S, H, D, order=order,
                                      stream_qk=sq, stream_v=sv if two else sq)
-                ms = time_graph_loop(torch, rotating, sq, n_sets, replays=10)
+                rounds = max(1, -(-32 // n_sets))      # at least 32 calls per graph: a replay boundary breaks the chain of launches
+                ms = time_graph_loop(torch, rotating, sq, n_sets * rounds, replays=10)
                 if ms is None:
                     continue
                 out[name][oname]["back_to_back_rotating_buffers"] = {
-                    "us_per_layer": 1e3 * ms, "gbs": b / (ms * 1e-3) / 1e9, "buffer_sets": n_sets,
-                    "how": "one CUDA graph of buffer_sets consecutive calls, replayed 10 times between two events (median of 5)",
+                    "us_per_layer": 1e3 * ms, "gbs": b / (ms * 1e-3) / 1e9, "buffer_sets": n_sets, "calls_per_graph": n_sets * rounds,
+                    "how": "one CUDA graph of calls_per_graph consecutive calls walking the buffer sets, replayed 10 times between two events (median of 5)",
                     "working_set_bytes": n_sets * b, "exceeds_4x_l2": bool(n_sets * b >= 4 * 126e6)}
             del sets
         del q, k, v, qh, kh, vh
@@ -789,8 +790,8 @@ def temporal_rows(torch, binding, args):
                                        metric, mask, idx, na, *([None] * 3 if direct else cmp_), *cch, ws,
                                        binding.vmajor_workspace_bytes(P, S, H, D, T_),
                                        order=binding.LUMP, stream_qk=sq, stream_v=sq)
-        return time_graph_loop(torch, rotating, sq, 4, replays=10)
-    how = "one CUDA graph of 4 consecutive steps alternating between two buffer sets, replayed 10 times (median of 5)"
+        return time_graph_loop(torch, rotating, sq, 16, replays=5)
+    how = "one CUDA graph of 16 consecutive steps alternating between two buffer sets, replayed 5 times (median of 5)"
     ms = rotating_loop(T, n_groups)
     if ms is not None:
         out["steps_1_to_7_selective"]["back_to_back_rotating_buffers"] = {
