@@ -335,3 +335,38 @@ def test_calls_chained_on_one_stream_keep_their_order(P, S, H, D):
     assert int(na.item()) == n_units - n_cached
     assert np.array_equal(idx.cpu().numpy()[:n_units - n_cached], np.arange(n_cached, n_units))
     assert np.array_equal(u16(cache[2]).reshape(H, S, D), oracle.ulysses_a2a(L["v"], P))
+
+
+def test_chained_calls_replayed_as_a_cuda_graph_keep_their_order():
+    """The same dependent chain captured into a CUDA graph (the dependent launches become
+    programmatic edges of the graph) and replayed: still the input, bit for bit."""
+    P, S, H, D = 4, 2048, 8, 128
+    L, _ = _layer(P, S, H, D, seed=13)
+    E = S * H * D
+    x0 = [dev(L[n]) for n in "qkv"]
+    seq = [[torch.zeros(E, dtype=torch.int16, device="cuda") for _ in range(3)] for _ in range(2)]
+    head = [[torch.zeros(E, dtype=torch.int16, device="cuda") for _ in range(3)] for _ in range(2)]
+    st = torch.cuda.Stream()
+
+    def chain():
+        src = x0
+        for i in range(4):
+            order = binding.V_FIRST if i % 2 == 0 else binding.LUMP
+            binding.ulysses_a2a(*src, *head[i % 2], P, S, H, D, order=order, stream_qk=st, stream_v=st)
+            binding.ulysses_a2a_inverse(*head[i % 2], *seq[i % 2], P, S, H, D, stream=st)
+            src = seq[i % 2]
+        return src
+    chain()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        last = chain()
+    for t in seq[0] + seq[1] + head[0] + head[1]:
+        t.zero_()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(st):
+        g.replay()
+        g.replay()
+    st.synchronize()
+    for n, got in zip("qkv", last):
+        assert np.array_equal(u16(got).reshape(S, H, D), L[n]), n
